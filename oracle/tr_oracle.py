@@ -1,0 +1,259 @@
+"""CPU oracle for one Token Recycling verify-and-recycle step.
+
+TEST INFRASTRUCTURE ONLY.  This module is the slow, plain definition that the
+CUDA path is checked against.  It shares no code with the CUDA path and is
+imported only by the tests, by the smoke check and by the benchmark's
+``cpu_baseline`` / ``--impl reference`` legs.  The product path never calls it.
+
+Everything is written in the paper's order and notation:
+
+  V      vocabulary size                       (Sec. 3.1)
+  k      candidates stored per token           (Sec. 3.1)
+  M      adjacency matrix, int [V, k]          (Sec. 3.1)
+  Tree   static template: parent[i], rank[i]   (Sec. 3.2, Appendix "Draft Tree
+         Algorithm and Structure", Algorithm 1)
+  S      merged sequence = tree tokens in layer (BFS) order, root first
+                                               (Sec. 3.3, Algorithm 1)
+  O      per-node argtopk of the output distribution (Appendix "Explanation of
+         Three Update Strategies")
+
+Floating point: attention is evaluated in float64 from the given inputs.
+Top-k only compares float32 values, so it is exact.
+
+Pin status (tests/test_oracle_pins.py): every function below is pinned by a
+test that does not re-use its own formula; see each docstring.  The whole step
+has no printed numeric example in the paper, so `step` is pinned only through
+its parts and through the losslessness property (Sec. 1, Sec. 2.2).
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+# --------------------------------------------------------------------------
+# Static tree template (Sec. 3.2 "static and imbalanced"; Appendix tree figure)
+# --------------------------------------------------------------------------
+def template_from_branching(b, max_nodes):
+    """Build a static, left-heavy tree template in layer order.
+
+    The paper's own tree is given only as a figure; the workload definition
+    used here generates one by rule: a node at depth d whose rank among its
+    siblings is r gets max(0, b[d] - r) children, children are appended parent
+    by parent with rank ascending, and the list is cut at `max_nodes`.  Depths
+    past the end of `b` re-use its last entry.  The rule reproduces the
+    properties Sec. 3.2 states: earlier nodes in a layer have more children and
+    reach deeper, and the number on a node is the column of M it is drawn from.
+
+    Returns (parent, rank): parent[0] = -1, rank[0] = 0.
+    Pinned by: node counts and per-level histograms worked out by hand
+    (1,8,10,20,25,16 for b=(8,4,3,2,2,1) cut at 80; 1,4,3,2,2,2,1 for
+    b=(4,2,1) cut at 15).
+    """
+    b = list(b)
+    parent, rank, depth = [-1], [0], [0]
+    head = 0
+    while head < len(parent) and len(parent) < max_nodes:
+        d = depth[head]
+        bd = b[min(d, len(b) - 1)]
+        for r in range(max(0, bd - rank[head])):
+            if len(parent) >= max_nodes:
+                break
+            parent.append(head)
+            rank.append(r)
+            depth.append(d + 1)
+        head += 1
+    return np.asarray(parent, dtype=np.int64), np.asarray(rank, dtype=np.int64)
+
+
+def node_depth(parent):
+    """Depth of every node (root = 0)."""
+    depth = np.zeros(len(parent), dtype=np.int64)
+    for i in range(1, len(parent)):
+        depth[i] = depth[parent[i]] + 1
+    return depth
+
+
+def ancestor_mask(parent):
+    """anc[i, j] is True iff j == i or j is an ancestor of i (Sec. 2.2: a node
+    attends to the nodes on its own root path, never to siblings)."""
+    n = len(parent)
+    anc = np.zeros((n, n), dtype=bool)
+    for i in range(n):
+        j = i
+        while j >= 0:
+            anc[i, j] = True
+            j = parent[j]
+    return anc
+
+
+# --------------------------------------------------------------------------
+# Tree attention (Sec. 2.2 "Tree Attention")
+# --------------------------------------------------------------------------
+def tree_attention(q, k, v, ctx_len, parent, scale=None):
+    """Masked attention of the tree's queries over prefix + tree keys.
+
+    q : [N, Hq, D]        queries of the N tree nodes
+    k : [Hkv, C + N, D]   keys; rows 0..C-1 are the prefix, rows C..C+N-1 the
+    v : [Hkv, C + N, D]   tree nodes in the same order as q
+    Node i sees every prefix row and tree row j iff j is i or an ancestor of i.
+    Query head h uses KV head h // (Hq // Hkv).
+    Returns float64 [N, Hq, D].
+
+    Pinned by: equality with plain causal attention run separately over
+    prefix + each root-to-leaf path; closed forms (equal keys -> mean of the
+    visible values; one dominating key -> that value row); N = 1 against a
+    library attention routine.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    k = np.asarray(k, dtype=np.float64)
+    v = np.asarray(v, dtype=np.float64)
+    n, hq, d = q.shape
+    hkv = k.shape[0]
+    c = int(ctx_len)
+    group = hq // hkv
+    if scale is None:
+        scale = 1.0 / np.sqrt(d)
+    anc = ancestor_mask(parent)
+    visible = np.concatenate([np.ones((n, c), dtype=bool), anc], axis=1)  # [N, C+N]
+    out = np.zeros((n, hq, d), dtype=np.float64)
+    for h in range(hq):
+        g = h // group
+        s = (q[:, h, :] @ k[g, : c + n, :].T) * scale        # [N, C+N]
+        s = np.where(visible, s, -np.inf)
+        s = s - s.max(axis=1, keepdims=True)
+        p = np.exp(s)                                         # masked -> exactly 0
+        p = p / p.sum(axis=1, keepdims=True)
+        out[:, h, :] = p @ v[g, : c + n, :]
+    return out
+
+
+# --------------------------------------------------------------------------
+# argtopk (Sec. 2.1)
+# --------------------------------------------------------------------------
+def argtopk(logits, k):
+    """Indices of the k largest entries of every row, largest first; equal
+    values are ordered by lower index first (the argmax convention the paper's
+    appendix on identical probabilities describes, applied at every rank).
+    Column 0 is therefore the argmax (Sec. 2.1: x^0 = x).
+
+    Definition written out: sort the whole row, keep the first k.
+    Pinned by: pure-Python brute force on tie-heavy rows, hand cases with
+    -inf / signed zeros, agreement with a library top-k on tie-free rows.
+    """
+    logits = np.asarray(logits, dtype=np.float32)
+    n, v = logits.shape
+    out = np.zeros((n, k), dtype=np.int64)
+    for i in range(n):
+        # stable sort of the negated row: descending value, ascending index on ties
+        order = np.argsort(-logits[i], kind="stable")
+        out[i] = order[:k]
+    return out
+
+
+# --------------------------------------------------------------------------
+# Verification (Sec. 2.2 "Guess and Verify", Sec. 3.3)
+# --------------------------------------------------------------------------
+def accept(S, argmax, parent):
+    """Longest correct path of the draft tree.
+
+    A tree node c is correct iff its parent is correct and its token equals the
+    model's greedy token after the parent, S[c] == argmax[parent[c]]; the root
+    (last confirmed token) is correct by definition.  The deepest correct node
+    wins, the lowest layer-order index among equally deep ones.  The step emits
+    the accepted draft tokens plus one more greedy token taken at the last
+    accepted node, so between 1 and depth_max + 1 tokens.
+
+    Returns (n_new, acc_nodes, out_tokens, next_root).
+    Pinned by: brute force over all root-to-node paths; losslessness against
+    token-by-token greedy decoding of a toy model.
+    """
+    S = np.asarray(S)
+    n = len(S)
+    depth = node_depth(parent)
+    valid = np.zeros(n, dtype=bool)
+    valid[0] = True
+    for c in range(1, n):
+        valid[c] = valid[parent[c]] and (S[c] == argmax[parent[c]])
+    best = 0
+    for c in range(n):
+        if valid[c] and depth[c] > depth[best]:
+            best = c
+    path = []
+    c = best
+    while c >= 0:
+        path.append(c)
+        c = parent[c]
+    acc_nodes = path[::-1]
+    out_tokens = [int(S[c]) for c in acc_nodes[1:]] + [int(argmax[best])]
+    return len(out_tokens), acc_nodes, out_tokens, int(argmax[best])
+
+
+# --------------------------------------------------------------------------
+# Matrix update (Sec. 3.3; Appendix "Explanation of Three Update Strategies")
+# --------------------------------------------------------------------------
+def update_matrix(M, S, O):
+    """M[S[i]] <- O[i] for every node of the merged sequence, root and rejected
+    nodes included, applied in increasing i: a token that occurs several times
+    keeps the row of its last occurrence (the appendix's "Last" strategy, which
+    is one of the outcomes the uncontrolled parallel update may produce).
+    In place; also returns M.
+    Pinned by: the appendix's worked example S = [a, b, c, a, d].
+    """
+    for i in range(len(S)):
+        M[S[i], :] = O[i, :]
+    return M
+
+
+# --------------------------------------------------------------------------
+# Draft tree retrieval (Sec. 3.2, Algorithm 1)
+# --------------------------------------------------------------------------
+def bfs_tree(M, parent, rank, root):
+    """Merged sequence S for the next step.
+
+    Algorithm 1, with the depth counter advancing once per iteration: the
+    current layer L starts as (root); xs = M[L] holds all candidates of the
+    layer; the template picks from the flattened xs the entries
+    (position of the parent inside L) * k + rank for each child; S collects the
+    layers in order.
+    Pinned by: the two-layer walk-through of Sec. 3.2 on symbolic tokens; node
+    count and parent structure; all-zero matrix -> all drafts are token 0.
+    """
+    parent = np.asarray(parent)
+    rank = np.asarray(rank)
+    n = len(parent)
+    k = M.shape[1]
+    depth = node_depth(parent)
+    S = []
+    L = np.asarray([root], dtype=np.int64)
+    layer_nodes = [0]                         # template nodes forming layer L
+    d = 0
+    while len(S) < n:
+        S.extend(int(t) for t in L)
+        xs = M[L]                             # [|L|, k]
+        nxt = [i for i in range(n) if depth[i] == d + 1]
+        pos = {node: p for p, node in enumerate(layer_nodes)}
+        index = [pos[parent[i]] * k + rank[i] for i in nxt]   # Tree[d].index
+        L = xs.reshape(-1)[index] if index else np.zeros(0, dtype=np.int64)
+        layer_nodes = nxt
+        d += 1
+        if not nxt:
+            break
+    return np.asarray(S, dtype=np.int64)
+
+
+# --------------------------------------------------------------------------
+# One whole step
+# --------------------------------------------------------------------------
+def verify_update(M, S, logits, parent, rank):
+    """argtopk -> accept -> update M -> next tree from the updated M, rooted at
+    the last confirmed token (the retrieve / verify / update cycle of Sec. 3 and
+    Sec. 5.4).  M is modified in place.
+    Returns dict(topk, n_new, acc_nodes, out_tokens, next_root, next_tree).
+    """
+    k = M.shape[1]
+    O = argtopk(logits, k)
+    n_new, acc_nodes, out_tokens, next_root = accept(S, O[:, 0], parent)
+    update_matrix(M, S, O)
+    nxt = bfs_tree(M, parent, rank, next_root)
+    return dict(topk=O, n_new=n_new, acc_nodes=acc_nodes, out_tokens=out_tokens,
+                next_root=next_root, next_tree=nxt)

@@ -1,0 +1,370 @@
+"""Pins for the CPU oracle: each check uses something other than the oracle's
+own formula - values the paper prints, closed forms, brute force, a library
+routine on a special case - so that a wrong sign, index or dropped term fails."""
+import itertools
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tr_oracle as orc
+from paper_2408_08696_b200 import synth
+
+
+def _read_golden(path):
+    rows = {}
+    for line in open(path):
+        line = line.strip()
+        if not line or line.startswith("#"):
+            continue
+        key, val = line.split(":", 1)
+        rows[key.strip()] = [int(x) for x in val.split()]
+    return rows
+
+
+# ---------------------------------------------------------------- template
+def test_template_level_histograms(golden_dir):
+    for line in open(os.path.join(golden_dir, "template_levels.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        parts = [p.split(":")[1].split() for p in line.split("|")]
+        b, max_nodes, levels = [int(x) for x in parts[0]], int(parts[1][0]), [int(x) for x in parts[2]]
+        parent, rank = orc.template_from_branching(b, max_nodes)
+        assert len(parent) == max_nodes
+        depth = orc.node_depth(parent)
+        assert np.bincount(depth).tolist() == levels
+
+
+def test_template_structure_is_layer_ordered_and_left_heavy():
+    parent, rank = orc.template_from_branching((8, 4, 3, 2, 2, 1), 80)
+    depth = orc.node_depth(parent)
+    assert parent[0] == -1 and rank[0] == 0
+    assert all(parent[i] < i for i in range(1, 80))
+    assert all(depth[i] <= depth[i + 1] for i in range(79))          # layer order
+    assert all(parent[i] <= parent[i + 1] for i in range(1, 79))     # parent by parent
+    # siblings: ranks 0,1,2.. in order
+    for p in range(80):
+        kids = [i for i in range(80) if parent[i] == p]
+        assert [rank[i] for i in kids] == list(range(len(kids)))
+    # imbalance (Sec. 3.2): earlier siblings never have fewer children than later ones
+    nchild = np.bincount(parent[1:], minlength=80)
+    for p in range(80):
+        kids = [i for i in range(80) if parent[i] == p]
+        full = [i for i in kids if depth[i] < 4]       # away from the truncated last level
+        assert all(nchild[a] >= nchild[b] for a, b in zip(full, full[1:]))
+    # paper: maximum acceptance length 6 with 6 layers -> deepest node at depth 5 (+1 bonus token)
+    assert depth.max() + 1 == 6
+    assert rank.max() < 8
+
+
+def test_storage_matches_table_2():
+    # Table 2 / Sec. 4.1: k=8 costs 1.95 MB (< 2 MB): V*k entries; 8-byte ids give 1.953 MiB,
+    # the int32 matrix of this build is half of that.
+    V, k = 32000, 8
+    M = np.zeros((V, k), dtype=np.int32)
+    assert M.size == V * k
+    assert abs(V * k * 8 / 2**20 - 1.95) < 0.01
+    assert M.nbytes == 1_024_000 and M.nbytes < 2 * 2**20
+
+
+# ---------------------------------------------------------------- argtopk
+def _brute_topk(row, k):
+    idx = list(range(len(row)))
+    chosen = []
+    for _ in range(k):
+        best = None
+        for i in idx:
+            if i in chosen:
+                continue
+            if best is None or row[i] > row[best]:      # strict: first (lowest) index wins ties
+                best = i
+        chosen.append(best)
+    return chosen
+
+
+def test_topk_bruteforce_ties():
+    rng = np.random.default_rng(1)
+    for trial in range(20):
+        v = int(rng.integers(8, 60))
+        x = rng.integers(-3, 4, size=(5, v)).astype(np.float32)       # heavy ties
+        got = orc.argtopk(x, 8)
+        for i in range(5):
+            assert got[i].tolist() == _brute_topk(x[i].tolist(), 8)
+
+
+def test_topk_special_values():
+    ninf = -np.inf
+    x = np.array([[ninf, 0.0, -0.0, 5.0, ninf, 5.0, -1.0, 0.0, 2.0]], dtype=np.float32)
+    # 5.0@3, 5.0@5, 2.0@8, zeros (signed zeros compare equal -> index order 1,2,7), -1@6, -inf@0
+    assert orc.argtopk(x, 8)[0].tolist() == [3, 5, 8, 1, 2, 7, 6, 0]
+    assert orc.argtopk(np.zeros((1, 20), np.float32), 8)[0].tolist() == list(range(8))
+
+
+def test_topk_column0_is_argmax_and_matches_library_without_ties():
+    rng = np.random.default_rng(2)
+    x = rng.standard_normal((16, 5000)).astype(np.float32)
+    got = orc.argtopk(x, 8)
+    assert (got[:, 0] == x.argmax(axis=1)).all()                   # Sec. 2.1: x^0 = argmax
+    lib = torch.topk(torch.from_numpy(x), 8, dim=1).indices.numpy()
+    assert (got == lib).all()
+    vals = np.take_along_axis(x, got, axis=1)
+    assert (np.diff(vals, axis=1) <= 0).all()
+
+
+# ---------------------------------------------------------------- attention
+def _causal_path_attention(q_path, k_all, v_all, scale):
+    """Plain causal attention of one linear sequence: prefix rows then the path
+    rows; query t sees the prefix and path rows 0..t.  Pure Python loops."""
+    out = []
+    c = k_all.shape[0] - q_path.shape[0]
+    for t in range(q_path.shape[0]):
+        ks = k_all[: c + t + 1]
+        vs = v_all[: c + t + 1]
+        s = [float(np.dot(q_path[t], kk)) * scale for kk in ks]
+        m = max(s)
+        e = [np.exp(si - m) for si in s]
+        z = sum(e)
+        out.append(sum(ei / z * vi for ei, vi in zip(e, vs)))
+    return np.stack(out)
+
+
+@pytest.mark.parametrize("hq,hkv", [(2, 2), (4, 2)])
+def test_tree_attention_equals_per_path_causal(hq, hkv):
+    rng = np.random.default_rng(3)
+    parent, rank = orc.template_from_branching((3, 2, 1), 9)
+    n, d, c = len(parent), 8, 5
+    q = rng.standard_normal((n, hq, d))
+    k = rng.standard_normal((hkv, c + n, d))
+    v = rng.standard_normal((hkv, c + n, d))
+    out = orc.tree_attention(q, k, v, c, parent)
+    scale = 1 / np.sqrt(d)
+    leaves = [i for i in range(n) if i not in set(parent.tolist())]
+    covered = set()
+    for leaf in leaves:
+        path = []
+        j = leaf
+        while j >= 0:
+            path.append(j)
+            j = parent[j]
+        path = path[::-1]
+        for h in range(hq):
+            g = h // (hq // hkv)
+            k_lin = np.concatenate([k[g, :c], k[g, c + np.array(path)]])
+            v_lin = np.concatenate([v[g, :c], v[g, c + np.array(path)]])
+            ref = _causal_path_attention(q[path, h], k_lin, v_lin, scale)
+            np.testing.assert_allclose(out[path, h], ref, rtol=1e-12, atol=1e-12)
+        covered.update(path)
+    assert covered == set(range(n))
+
+
+def test_tree_attention_needs_self_key():
+    # Root with no prefix sees only itself: output must be exactly its own value row.
+    parent = np.array([-1, 0, 0])
+    rng = np.random.default_rng(4)
+    q, k, v = rng.standard_normal((3, 1, 4)), rng.standard_normal((1, 3, 4)), rng.standard_normal((1, 3, 4))
+    out = orc.tree_attention(q, k, v, 0, parent)
+    np.testing.assert_allclose(out[0, 0], v[0, 0], rtol=1e-14)
+    # siblings 1 and 2 never see each other: changing node 2's key/value leaves node 1 unchanged
+    k2, v2 = k.copy(), v.copy()
+    k2[0, 2] += 5.0
+    v2[0, 2] -= 7.0
+    out2 = orc.tree_attention(q, k2, v2, 0, parent)
+    np.testing.assert_array_equal(out[1], out2[1])
+    assert not np.allclose(out[2], out2[2])
+
+
+def test_tree_attention_closed_forms():
+    parent, _ = orc.template_from_branching((2, 2), 7)
+    n, d, c = 7, 6, 4
+    rng = np.random.default_rng(5)
+    q = rng.standard_normal((n, 1, d))
+    v = rng.standard_normal((1, c + n, d))
+    # all keys equal -> uniform weights over the visible set -> mean of visible values
+    k = np.tile(rng.standard_normal((1, 1, d)), (1, c + n, 1))
+    out = orc.tree_attention(q, k, v, c, parent)
+    anc = orc.ancestor_mask(parent)
+    for i in range(n):
+        vis = list(range(c)) + [c + j for j in range(n) if anc[i, j]]
+        np.testing.assert_allclose(out[i, 0], v[0, vis].mean(axis=0), rtol=1e-12)
+    # one dominating key (a prefix row aligned with every query) -> that value row
+    k = np.zeros((1, c + n, d))
+    q = np.ones((n, 1, d))
+    k[0, 2] = 1000.0
+    out = orc.tree_attention(q, k, v, c, parent)
+    np.testing.assert_allclose(out[:, 0], np.tile(v[0, 2], (n, 1)), rtol=1e-9)
+
+
+def test_tree_attention_single_node_is_library_decode():
+    rng = np.random.default_rng(6)
+    d, c, h = 16, 33, 3
+    q = rng.standard_normal((1, h, d)).astype(np.float32)
+    k = rng.standard_normal((h, c + 1, d)).astype(np.float32)
+    v = rng.standard_normal((h, c + 1, d)).astype(np.float32)
+    out = orc.tree_attention(q, k, v, c, np.array([-1]))
+    ref = torch.nn.functional.scaled_dot_product_attention(
+        torch.from_numpy(q).permute(1, 0, 2), torch.from_numpy(k), torch.from_numpy(v))
+    np.testing.assert_allclose(out[0], ref[:, 0].numpy(), rtol=2e-5, atol=2e-6)
+
+
+def test_tree_attention_gqa_head_mapping():
+    rng = np.random.default_rng(7)
+    parent, _ = orc.template_from_branching((2, 1), 4)
+    q = rng.standard_normal((4, 4, 8))
+    k, v = rng.standard_normal((2, 7, 8)), rng.standard_normal((2, 7, 8))
+    out = orc.tree_attention(q, k, v, 3, parent)
+    for h in range(4):
+        one = orc.tree_attention(q[:, h:h + 1], k[h // 2:h // 2 + 1], v[h // 2:h // 2 + 1], 3, parent)
+        np.testing.assert_allclose(out[:, h], one[:, 0], rtol=1e-13)
+
+
+# ---------------------------------------------------------------- accept
+def _brute_accept(S, argmax, parent):
+    n = len(S)
+    best_len, best_leaf = 0, 0
+    for leaf in range(n):
+        path, j = [], leaf
+        while j >= 0:
+            path.append(j)
+            j = parent[j]
+        path = path[::-1]
+        ok = all(S[c] == argmax[parent[c]] for c in path[1:])
+        if ok and len(path) - 1 > best_len:
+            best_len, best_leaf = len(path) - 1, leaf
+    return best_len + 1, best_leaf
+
+
+def test_accept_bruteforce_including_duplicates():
+    rng = np.random.default_rng(8)
+    parent, _ = orc.template_from_branching((4, 2, 1), 15)
+    for trial in range(300):
+        S = rng.integers(0, 3, size=15)
+        am = rng.integers(0, 3, size=15)
+        n_new, acc, toks, nxt = orc.accept(S, am, parent)
+        bn, bleaf = _brute_accept(S, am, parent)
+        assert n_new == bn and acc[-1] == bleaf and acc[0] == 0
+        assert 1 <= n_new <= orc.node_depth(parent).max() + 1
+        assert toks[-1] == am[acc[-1]] == nxt
+        assert toks[:-1] == [S[c] for c in acc[1:]]
+
+
+def test_accept_nothing_matches_gives_one_token():
+    parent, _ = orc.template_from_branching((4, 2, 1), 15)
+    S = np.arange(15) + 100
+    am = np.arange(15)
+    assert orc.accept(S, am, parent) == (1, [0], [0], 0)      # AR step: MAT counts the bonus token
+
+
+def _toy_logits(path_tokens, V, salt):
+    """Deterministic toy model: logits are a pure function of the token path."""
+    h = salt
+    for t in path_tokens:
+        h = (h * 1000003 + int(t) + 12345) % (2**61 - 1)
+    return np.random.default_rng(h).standard_normal(V).astype(np.float32)
+
+
+@pytest.mark.parametrize("init", ["zero", "random"])
+def test_losslessness_against_greedy_decoding(init):
+    """Sec. 1 / Sec. 2.2: speculative decoding with verification emits exactly the
+    greedy sequence, whatever the matrix and template hold."""
+    V, k, steps = 50, 4, 25
+    parent, rank = orc.template_from_branching((3, 2, 1), 10)
+    rng = np.random.default_rng(9)
+    M = np.zeros((V, k), dtype=np.int64) if init == "zero" else rng.integers(0, V, size=(V, k))
+    prefix = [7]
+    ar = list(prefix)
+    for _ in range(steps * 4 + 4):
+        ar.append(int(np.argmax(_toy_logits(ar, V, 5))))
+    seq = list(prefix)
+    S = orc.bfs_tree(M, parent, rank, seq[-1])
+    mats = []
+    for _ in range(steps):
+        logits = np.zeros((len(parent), V), dtype=np.float32)
+        for i in range(len(parent)):
+            path, j = [], i
+            while j > 0:
+                path.append(int(S[j]))
+                j = parent[j]
+            logits[i] = _toy_logits(seq + path[::-1], V, 5)
+        r = orc.verify_update(M, S, logits, parent, rank)
+        assert S[0] == seq[-1]
+        seq += r["out_tokens"]
+        assert r["next_tree"][0] == seq[-1]
+        S = r["next_tree"]
+        mats.append(r["n_new"])
+        assert ((M >= 0) & (M < V)).all()
+    assert seq == ar[: len(seq)]
+    assert max(mats) > 1            # recycling does accept drafts on this toy model
+
+
+# ---------------------------------------------------------------- update
+def test_update_last_writer_matches_appendix_example(golden_dir):
+    g = _read_golden(os.path.join(golden_dir, "update_last_example.txt"))
+    S = np.array(g["S"])
+    O = np.array([g["O%d" % i] for i in range(5)])
+    M = np.full((20, 4), -1, dtype=np.int64)
+    orc.update_matrix(M, S, O)
+    assert M[10].tolist() == g["M[a] last"] != g["M[a] first"]
+    assert M[11].tolist() == g["M[b]"] and M[12].tolist() == g["M[c]"] and M[13].tolist() == g["M[d]"]
+    untouched = [i for i in range(20) if i not in (10, 11, 12, 13)]
+    assert (M[untouched] == -1).all()
+
+
+def test_update_covers_root_and_rejected_nodes():
+    # Sec. 3.3 / Sec. 5.2 "Effect of Rejected Tokens": every node of S gets its row, not only accepted ones.
+    parent, rank = orc.template_from_branching((2, 1), 4)
+    V, k = 30, 2
+    M = np.zeros((V, k), dtype=np.int64)
+    S = np.array([5, 6, 7, 8])
+    logits = np.full((4, V), -1.0, dtype=np.float32)
+    for i in range(4):
+        logits[i, 20 + i] = 3.0
+        logits[i, 10 + i] = 2.0
+    r = orc.verify_update(M, S, logits, parent, rank)
+    assert r["n_new"] == 1                                    # nothing accepted
+    for i, t in enumerate(S):
+        assert M[t].tolist() == [20 + i, 10 + i]
+
+
+# ---------------------------------------------------------------- BFS
+def test_bfs_matches_section_3_2_walkthrough(golden_dir):
+    g = _read_golden(os.path.join(golden_dir, "bfs_walkthrough.txt"))
+    M = np.zeros((11, 3), dtype=np.int64)
+    for t in (1, 2, 3):
+        M[t] = g["M[%d]" % t]
+    S = orc.bfs_tree(M, np.array(g["parent"]), np.array(g["rank"]), g["root"][0])
+    assert S.tolist() == g["S"]
+
+
+def test_bfs_node_count_parent_structure_and_zero_matrix():
+    parent, rank = orc.template_from_branching((8, 4, 3, 2, 2, 1), 80)
+    rng = np.random.default_rng(10)
+    V, k = 500, 8
+    M = rng.integers(0, V, size=(V, k))
+    S = orc.bfs_tree(M, parent, rank, 17)
+    assert len(S) == 80 and S[0] == 17
+    for i in range(1, 80):                                    # per-node statement of Algorithm 1
+        assert S[i] == M[S[parent[i]], rank[i]]
+    Z = orc.bfs_tree(np.zeros((V, k), dtype=np.int64), parent, rank, 17)
+    assert Z[0] == 17 and (Z[1:] == 0).all()                  # Sec. 3.1: zero init -> no valid candidates yet
+
+
+# ---------------------------------------------------------------- generators
+def test_synth_is_seeded_and_shaped():
+    w = synth.WORKLOADS["tiny"]
+    a, b = synth.noise_logits(w, 2), synth.noise_logits(w, 2)
+    assert a.shape == (2, 1, 15, 1000) and (a == b).all()
+    succ = synth.zipf_successors(w)
+    assert succ.min() >= 0 and succ.max() < w.vocab
+    assert (succ < 10).mean() > 0.3                            # Zipf(1.1): mass on the first ranks
+    q, k, v = synth.attention_inputs(w)
+    assert q.shape == (1, 1, 15, 4, 64) and k.shape == (1, 1, 4, 143, 64)
+    pool = synth.normal_pool(w.seed)
+    qs, ks, vs = synth.attention_slice(w, pool, 0, 0, 2)
+    assert (ks == k[0, 0, 2]).all() and (vs == v[0, 0, 2]).all() and (qs == q[0, 0]).all()
+    x = np.array([1.0, 1.00390625, -2.5, 3.1415926], dtype=np.float32)
+    ref = torch.from_numpy(x).to(torch.bfloat16).to(torch.float32).numpy()
+    assert (synth.bf16_bits_to_f32(synth.f32_to_bf16_bits(x)) == ref).all()
+    lg = synth.step_logits(a[0, 0], np.zeros(15, dtype=np.int64), succ, 4.0)
+    assert np.count_nonzero(lg != a[0, 0]) == 15
+    assert len(synth.WORKLOADS["llama2-70b-b8"].ctx) == 8
