@@ -1,0 +1,184 @@
+/*
+ * tr.h - C ABI of the Token Recycling (TR) verify-and-recycle step for one NVIDIA B200 (sm_100a).
+ *
+ * One TR decoding step (paper Sec. 3 and Sec. 5.4) is
+ *     retrieve a draft tree from the adjacency matrix   -> tr_build_tree
+ *     model forward with tree attention                  -> tr_tree_attention (attention only)
+ *     verify (argmax per node, longest correct path),
+ *     update the matrix with every node's top-k,
+ *     retrieve the next tree                             -> tr_verify_update
+ *
+ * Conventions
+ *   - Every pointer is marked HOST or DEVICE.  DEVICE pointers are caller-owned (for example PyTorch
+ *     tensors) unless stated; the library never frees them.
+ *   - `stream` is a cudaStream_t passed as void*; NULL is the legacy default stream.
+ *   - All entry points return a tr_status; none throws, aborts or synchronises the device unless its
+ *     comment says so.  Argument errors are detected on the host before any launch.
+ *   - tr_build_tree, tr_tree_attention and tr_verify_update allocate nothing, read nothing back and do
+ *     not synchronise, so they can be recorded in a CUDA graph.
+ *   - Anomalies only the device can see (a token id outside [0, vocab)) set a sticky bit in a flag word
+ *     (tr_device_flags); the offending access is skipped or clamped.  Kernels never trap.
+ *   - Notation follows the paper: V = vocabulary size, k = candidates per token, M = adjacency matrix
+ *     [V, k], S = merged sequence (tree tokens in layer order, root first), N = tree nodes incl. root.
+ */
+#ifndef TR_H_
+#define TR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tr_ctx tr_ctx; /* opaque; owns M, the template tables and the kernels' scratch */
+
+typedef int32_t tr_status;
+#define TR_OK 0
+#define TR_ERR_INVALID_ARG (-1)
+#define TR_ERR_TEMPLATE (-2)
+#define TR_ERR_UNSUPPORTED (-3)
+#define TR_ERR_CUDA (-4)
+#define TR_ERR_NOMEM (-5)
+#define TR_ERR_DEVICE_FLAG (-6)
+
+#define TR_MAX_NODES 128 /* ancestor masks are 128-bit */
+#define TR_MAX_K 16
+
+/* Device flag bits (tr_device_flags). */
+#define TR_FLAG_BAD_TOKEN 1u    /* a tree/root token id was outside [0, V): row skipped / id clamped to 0 */
+#define TR_FLAG_WAIT_TIMEOUT 2u /* a bounded wait inside a kernel ran out (should never happen) */
+
+const char* tr_status_string(tr_status s);
+
+/*
+ * Static tree template by rule (Sec. 3.2: static, imbalanced - earlier siblings get more children).
+ * A node at depth d whose rank among its siblings is r gets max(0, b[min(d, nb-1)] - r) children; children
+ * are appended parent by parent, rank ascending (layer order), and the list is cut at max_nodes.
+ * HOST in: b[nb].  HOST out: parent_out[max_nodes], rank_out[max_nodes] (parent[0] = -1), *n_out = node count.
+ * Errors: TR_ERR_INVALID_ARG on NULL / non-positive sizes / max_nodes > TR_MAX_NODES.
+ */
+tr_status tr_template_from_branching(const int32_t* b, int32_t nb, int32_t max_nodes,
+                                     int32_t* parent_out, int32_t* rank_out, int32_t* n_out);
+
+/*
+ * Create a context on `device` (Sec. 3.1): allocates `batch` adjacency matrices M[V, k] (int32, zeroed: the
+ * paper's cold start), uploads the template and the tables derived from it (depth, ancestor bitmasks),
+ * and allocates the scratch the kernels need.  Synchronises once.
+ * HOST in: parent[n_nodes], rank[n_nodes] - the static tree in layer order: parent[0] = -1, 0 <= parent[i] < i,
+ *   depth non-decreasing, 0 <= rank[i] < k (rank = the column of M a node is drawn from, Appendix tree figure).
+ * Errors: TR_ERR_INVALID_ARG (vocab < k, k < 1 or > TR_MAX_K, batch < 1, NULL), TR_ERR_TEMPLATE
+ *   (malformed tree, n_nodes > TR_MAX_NODES), TR_ERR_CUDA / TR_ERR_NOMEM.
+ */
+tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32_t* parent, const int32_t* rank,
+                  int32_t n_nodes, int32_t batch, int32_t device);
+tr_status tr_destroy(tr_ctx* ctx); /* frees everything tr_init allocated; synchronises */
+
+/* Matrix state (Sec. 3.1: zero initialisation, or "hot start" = keep / restore an earlier matrix). */
+tr_status tr_matrix_zero(tr_ctx* ctx, void* stream);                                /* all sequences */
+tr_status tr_matrix_import(tr_ctx* ctx, int32_t seq, const int32_t* host_M);        /* HOST [V*k]; synchronises */
+tr_status tr_matrix_export(tr_ctx* ctx, int32_t seq, int32_t* host_M);              /* HOST [V*k]; synchronises */
+int32_t* tr_matrix_device_ptr(tr_ctx* ctx, int32_t seq);                            /* DEVICE, borrowed; NULL on error */
+
+/*
+ * Draft tree retrieval (Sec. 3.2, Algorithm 1): for every sequence b, tree[b][0] = root[b] and
+ * tree[b][i] = M_b[tree[b][parent[i]]][rank[i]], layer by layer.
+ * DEVICE in: d_root[batch].  DEVICE out: d_tree[batch * N] (the merged sequence S per sequence).
+ * A root outside [0, V) sets TR_FLAG_BAD_TOKEN and is treated as token 0.
+ */
+tr_status tr_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, void* stream);
+
+/*
+ * Tree attention (Sec. 2.2): for every sequence b, layer l, query head h and tree node i,
+ *   out[b,l,i,h,:] = softmax_j( scale * q[b,l,i,h,:] . k[b,l,g,j,:] ) @ v[b,l,g,j,:],  g = h / (Hq / Hkv),
+ * over the keys j in [0, C_b) (the prefix, all visible) and j = C_b + t for tree nodes t that are node i
+ * itself or one of its ancestors.  C_b = d_ctx_len[b]; the tree's K/V rows sit right after the prefix.
+ * bf16 inputs and output, fp32 accumulation.  Rows j >= C_b + N of the cache are never used, but rows below
+ * kv_rows may be fetched and must hold finite numbers.
+ *
+ * Addressing (strides in ELEMENTS; head_dim is contiguous):
+ *   q  : q   + b*q_stride[0]  + l*layer_stride_q  + h*q_stride[1]  + i*q_stride[2]
+ *   k,v: k   + b*kv_stride[0] + l*layer_stride_kv + g*kv_stride[1] + j*kv_stride[2]
+ *   out: out + b*o_stride[0]  + l*layer_stride_o  + h*o_stride[1]  + i*o_stride[2]
+ * All base pointers 16-byte aligned and all strides multiples of 8 elements.
+ * n_layers > 1 runs that many independent layers in one launch (layers of a real model are sequential;
+ * this is for callers that hold all layers' q already, e.g. benchmarks).
+ * Errors: TR_ERR_INVALID_ARG (NULL, bad head counts, alignment), TR_ERR_UNSUPPORTED (head_dim not 64/128).
+ */
+typedef struct {
+  const void* q;       /* DEVICE bf16 */
+  const void* k_cache; /* DEVICE bf16 */
+  const void* v_cache; /* DEVICE bf16 */
+  void* out;           /* DEVICE bf16 */
+  int32_t n_q_heads, n_kv_heads, head_dim;
+  const int32_t* d_ctx_len; /* DEVICE [batch] prefix lengths C_b, each <= max_ctx */
+  int32_t max_ctx;          /* upper bound of C_b, used for launch sizing */
+  int32_t kv_rows;          /* token rows addressable per (b, l, g) slice, >= max_ctx + N */
+  int64_t q_stride[3], kv_stride[3], o_stride[3]; /* (sequence, head, token) */
+  int32_t n_layers;
+  int64_t layer_stride_q, layer_stride_kv, layer_stride_o;
+  float scale;    /* 0 -> 1/sqrt(head_dim) */
+  int32_t splits; /* 0 -> chosen by the library; >0 forces that many KV splits (testing) */
+} tr_attn_args;
+tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* args, void* stream);
+
+/*
+ * Verify, recycle and retrieve (Sec. 2.1 argtopk, Sec. 2.2 verification, Sec. 3.3 update, Algorithm 1):
+ *   topk[b,i,:]  = indices of the k largest logits of node i, largest first, equal values by lower index
+ *   acceptance   : node c is correct iff parent(c) is correct and tree[c] == topk[parent(c)][0]; the deepest
+ *                  correct node wins (lowest layer-order index among equals)
+ *   out_tokens   = tokens of the accepted path below the root, then topk[last accepted][0]; n_new = their count
+ *   M_b[tree[i]] = topk[i,:] for every node i in increasing i (a repeated token keeps its last row)
+ *   next_tree    = tr_build_tree on the updated M_b rooted at the last emitted token (= next_root)
+ * DEVICE in : d_logits [batch, N, V] fp32 row-major (no NaN), d_tree [batch, N].
+ * DEVICE out: d_topk_idx [batch,N,k], d_n_new [batch], d_acc_nodes [batch, depth_max+1] (unused tail = -1),
+ *             d_out_tokens [batch, depth_max+1] (unused tail = -1), d_next_root [batch], d_next_tree [batch,N].
+ *             d_next_tree may alias d_tree.  depth_max+1 = tr_max_new_tokens(ctx).
+ */
+typedef struct {
+  int32_t* d_topk_idx;
+  int32_t* d_n_new;
+  int32_t* d_acc_nodes;
+  int32_t* d_out_tokens;
+  int32_t* d_next_root;
+  int32_t* d_next_tree;
+} tr_step_out;
+tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const int32_t* d_tree, const tr_step_out* out,
+                           void* stream);
+int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appendix: maximum acceptance length) */
+
+/* Copies the sticky flag word to HOST and synchronises the device. */
+tr_status tr_device_flags(tr_ctx* ctx, uint32_t* host_flags);
+
+/*
+ * One whole step from HOST buffers (pinned memory recommended): copies this step's inputs to the device,
+ * runs tr_tree_attention over n_layers layers, then tr_verify_update, copies the results back and waits.
+ * The prefix K/V (rows [0, C_b)) and the current tree stay resident in device buffers the caller owns.
+ * HOST in : h_q [batch, L, N, Hq, D] bf16; h_tree_k / h_tree_v [batch, L, Hkv, N, D] bf16 (this step's tree
+ *           rows, written to cache rows C_b..C_b+N-1; h_ctx_len[batch] gives C_b); h_logits [batch, N, V] fp32.
+ * DEVICE  : a->q / a->out must be buffers of that shape (used as staging), a->k_cache / a->v_cache the caches
+ *           with kv_stride/layer_stride_kv as described above; d_logits_staging [batch,N,V]; d_tree [batch,N]
+ *           current tree (updated in place to the next tree); d_out as in tr_verify_update.
+ * HOST out: h_out [batch, L, N, Hq, D] bf16; h_n_new [batch]; h_out_tokens [batch, depth_max+1];
+ *           h_next_tree [batch, N].
+ * Synchronises `stream` before returning.
+ */
+typedef struct {
+  const void* h_q;
+  const void* h_tree_k;
+  const void* h_tree_v;
+  const float* h_logits;
+  const int32_t* h_ctx_len;
+  float* d_logits_staging;
+  int32_t* d_tree;
+  void* h_out;
+  int32_t* h_n_new;
+  int32_t* h_out_tokens;
+  int32_t* h_next_tree;
+} tr_host_io;
+tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_step_out* d_out, const tr_host_io* io,
+                       void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TR_H_ */

@@ -1,0 +1,146 @@
+// Acceptance, matrix update and next-tree retrieval in one kernel (paper Sec. 2.2 verification, Sec. 3.3
+// update, Sec. 3.2 / Algorithm 1 retrieval), plus the stand-alone retrieval kernel behind tr_build_tree.
+//
+// One CTA per sequence, one thread per tree node (N <= 128).
+//   accept : node c is correct iff every edge on its root path matches, S[x] == argmax[parent(x)]; each thread
+//            walks its own path (<= depth_max steps); the deepest correct node, lowest index among equals, is
+//            found with one packed-key maximum (warp reduce + shared memory).
+//   update : M[S[i]] <- topk[i] for all i; when a token repeats, only the highest i writes, which is what the
+//            sequential loop "for i: M[S[i]] = O[i]" leaves behind - deterministic, no write races.
+//   BFS    : S'[0] = argmax[last accepted]; level by level S'[i] = M[S'[parent i]][rank i], reading the rows
+//            written a moment ago by this same CTA (ordered by __syncthreads()).
+#include "tr_internal.cuh"
+
+constexpr int TAIL_THREADS = 128;
+
+__device__ __forceinline__ void bfs_expand(const int32_t* __restrict__ M, int V, int k, int n,
+                                           const int32_t* __restrict__ parent, const int32_t* __restrict__ rank,
+                                           const int32_t* __restrict__ level_off, int depth_max,
+                                           int32_t* s_tree /* shared [n], s_tree[0] set */, int tid) {
+  // one dependent round of gathers per level; every node of a level is looked up in parallel
+  for (int d = 1; d <= depth_max; ++d) {
+    __syncthreads();
+    const int lo = level_off[d], hi = level_off[d + 1];
+    const int i = lo + tid;
+    if (i < hi) s_tree[i] = __ldcg(M + static_cast<size_t>(s_tree[parent[i]]) * k + rank[i]);
+  }
+  __syncthreads();
+}
+
+__global__ void __launch_bounds__(TAIL_THREADS)
+tr_build_tree_kernel(const int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* __restrict__ parent,
+                     const int32_t* __restrict__ rank, const int32_t* __restrict__ level_off, int depth_max,
+                     const int32_t* __restrict__ root, int32_t* __restrict__ tree, uint32_t* __restrict__ flags) {
+  __shared__ int32_t s_tree[TR_MAX_NODES];
+  const int b = blockIdx.x, tid = threadIdx.x;
+  const int32_t* M = M_all + static_cast<size_t>(b) * V * k;
+  if (tid == 0) {
+    int32_t r = root[b];
+    if (r < 0 || r >= V) {
+      atomicOr(flags, TR_FLAG_BAD_TOKEN);
+      r = 0;
+    }
+    s_tree[0] = r;
+  }
+  bfs_expand(M, V, k, n, parent, rank, level_off, depth_max, s_tree, tid);
+  if (tid < n) tree[static_cast<size_t>(b) * n + tid] = s_tree[tid];
+}
+
+__global__ void __launch_bounds__(TAIL_THREADS)
+tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* __restrict__ parent,
+               const int32_t* __restrict__ rank, const int32_t* __restrict__ depth,
+               const int32_t* __restrict__ level_off, int depth_max, const int32_t* tree_in,
+               const int32_t* __restrict__ topk_idx, int32_t* __restrict__ n_new, int32_t* __restrict__ acc_nodes,
+               int32_t* __restrict__ out_tokens, int32_t* __restrict__ next_root, int32_t* tree_out,
+               uint32_t* __restrict__ flags) {
+  __shared__ int32_t s_S[TR_MAX_NODES];
+  __shared__ int32_t s_argmax[TR_MAX_NODES];
+  __shared__ int32_t s_tree[TR_MAX_NODES];
+  __shared__ uint32_t s_best[TAIL_THREADS / 32];
+  const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  int32_t* M = M_all + static_cast<size_t>(b) * V * k;
+  const int32_t* topk = topk_idx + static_cast<size_t>(b) * n * k;
+  const int W = depth_max + 1;
+
+  int32_t tok = 0;
+  bool tok_ok = false;
+  if (tid < n) {
+    tok = tree_in[static_cast<size_t>(b) * n + tid];
+    tok_ok = (tok >= 0 && tok < V);
+    if (!tok_ok) atomicOr(flags, TR_FLAG_BAD_TOKEN);
+    s_S[tid] = tok;
+    s_argmax[tid] = topk[tid * k];
+  }
+  __syncthreads();
+
+  // ---- accept: walk this node's root path
+  uint32_t keyv = 0;
+  if (tid < n) {
+    bool ok = true;
+    for (int x = tid; x > 0;) {
+      const int p = parent[x];
+      ok = ok && (s_S[x] == s_argmax[p]);
+      x = p;
+    }
+    // deeper first, then lower index; +1 keeps every valid key above the 0 of idle threads
+    if (ok) keyv = (static_cast<uint32_t>(depth[tid]) << 8 | static_cast<uint32_t>(255 - tid)) + 1u;
+  }
+  const uint32_t wbest = __reduce_max_sync(0xFFFFFFFFu, keyv);
+  if (lane == 0) s_best[warp] = wbest;
+  __syncthreads();
+  uint32_t best = 0;
+#pragma unroll
+  for (int w = 0; w < TAIL_THREADS / 32; ++w) best = max(best, s_best[w]);
+  const int leaf = 255 - static_cast<int>((best - 1u) & 0xFFu);
+  const int acc_len = static_cast<int>((best - 1u) >> 8);  // accepted drafts = depth of the leaf
+  const int32_t bonus = s_argmax[leaf];
+
+  if (tid == 0) {
+    n_new[b] = acc_len + 1;
+    next_root[b] = bonus;
+    int x = leaf;
+    for (int d = acc_len; d >= 0; --d) {  // fill the path backwards
+      acc_nodes[b * W + d] = x;
+      if (d > 0) out_tokens[b * W + d - 1] = s_S[x];
+      x = parent[x];
+    }
+    out_tokens[b * W + acc_len] = bonus;
+    for (int d = acc_len + 1; d < W; ++d) {
+      acc_nodes[b * W + d] = -1;
+      out_tokens[b * W + d] = -1;
+    }
+    s_tree[0] = bonus;
+  }
+
+  // ---- update: last occurrence of each token writes its whole row
+  if (tid < n && tok_ok) {
+    bool last = true;
+    for (int j = tid + 1; j < n; ++j) last = last && (s_S[j] != tok);
+    if (last) {
+      int32_t* dst = M + static_cast<size_t>(tok) * k;
+      const int32_t* src = topk + tid * k;
+      for (int c = 0; c < k; ++c) dst[c] = src[c];
+    }
+  }
+  // ---- retrieve the next tree from the updated matrix (bfs_expand starts with a __syncthreads())
+  bfs_expand(M, V, k, n, parent, rank, level_off, depth_max, s_tree, tid);
+  if (tid < n) tree_out[static_cast<size_t>(b) * n + tid] = s_tree[tid];
+}
+
+tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s) {
+  tr_build_tree_kernel<<<ctx->batch, TAIL_THREADS, 0, s>>>(ctx->d_M, ctx->vocab, ctx->k, ctx->n_nodes, ctx->d_parent,
+                                                           ctx->d_rank, ctx->d_level_off, ctx->depth_max, d_root,
+                                                           d_tree, ctx->d_flags);
+  TR_CUDA_TRY(cudaGetLastError());
+  return TR_OK;
+}
+
+tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s) {
+  tr_tail_kernel<<<ctx->batch, TAIL_THREADS, 0, s>>>(ctx->d_M, ctx->vocab, ctx->k, ctx->n_nodes, ctx->d_parent,
+                                                     ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
+                                                     d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes,
+                                                     out->d_out_tokens, out->d_next_root, out->d_next_tree,
+                                                     ctx->d_flags);
+  TR_CUDA_TRY(cudaGetLastError());
+  return TR_OK;
+}

@@ -1,0 +1,57 @@
+// Internal declarations shared by the translation units of libtr.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <vector>
+
+#include "tr.h"
+
+#define TR_CUDA_TRY(expr)                                  \
+  do {                                                     \
+    cudaError_t e__ = (expr);                              \
+    if (e__ != cudaSuccess) {                              \
+      tr_set_last_cuda_error(e__, #expr, __FILE__, __LINE__); \
+      return (e__ == cudaErrorMemoryAllocation) ? TR_ERR_NOMEM : TR_ERR_CUDA; \
+    }                                                      \
+  } while (0)
+
+void tr_set_last_cuda_error(cudaError_t e, const char* what, const char* file, int line);
+
+// Top-k of one logits row is computed by TOPK_SEG_ELEMS-wide segments, one CTA each.
+constexpr int TOPK_THREADS = 256;
+constexpr int TOPK_ELEMS_PER_THREAD = 16;
+constexpr int TOPK_SEG_ELEMS = TOPK_THREADS * TOPK_ELEMS_PER_THREAD;  // 4096
+
+// Split-KV attention partials: [slot][ATTN_PART_ROWS][D] fp32 + [slot][ATTN_PART_ROWS][2] (m, l).
+constexpr int ATTN_PART_ROWS = 128;
+constexpr int ATTN_MAX_PART_SLOTS = 1024;
+
+struct tr_ctx {
+  int device = 0;
+  int vocab = 0, k = 0, n_nodes = 0, batch = 0, depth_max = 0;
+  int sm_count = 148;
+  std::vector<int32_t> h_parent, h_rank, h_depth;
+  // device tables
+  int32_t* d_parent = nullptr;   // [N]
+  int32_t* d_rank = nullptr;     // [N]
+  int32_t* d_depth = nullptr;    // [N]
+  int32_t* d_level_off = nullptr;  // [depth_max + 2]: nodes of level d are [off[d], off[d+1])
+  uint32_t* d_anc = nullptr;     // [N][4] bit j of row i: j is i or an ancestor of i
+  int32_t* d_M = nullptr;        // [batch][V][k]
+  // scratch
+  unsigned long long* d_topk_part = nullptr;  // [batch*N][segs][k] packed (value, index) keys
+  unsigned int* d_topk_ticket = nullptr;      // [batch*N]
+  int topk_segs = 0;
+  float* d_attn_part_o = nullptr;   // [slots][128][128]
+  float* d_attn_part_ml = nullptr;  // [slots][128][2]
+  uint32_t* d_flags = nullptr;
+};
+
+// launchers (host functions defined next to their kernels)
+tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s);
+tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s);
+tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);
+tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
+tr_status tr_attention_mma_setup();
+int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys);

@@ -1,0 +1,91 @@
+"""Device-side set-up of a synthetic workload: uploads the seeded inputs, creates the context and drives the
+step through the C-ABI binding.  Plumbing only (allocation, copies, launches, CUDA graphs); used by the GPU
+tests, the smoke check and the benchmark."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as tr
+from . import synth
+
+
+def bf16_tensor(bits_u16, device):
+    """uint16 bit patterns (numpy) -> torch.bfloat16 tensor on `device`."""
+    return torch.from_numpy(np.ascontiguousarray(bits_u16).view(np.int16)).to(device).view(torch.bfloat16)
+
+
+class DeviceWorkload:
+    def __init__(self, w: synth.Workload, n_layers=None, device=0, n_rot=4, with_attention=True, splits=0,
+                 zero_matrix=False):
+        self.w = w
+        self.dev = torch.device("cuda", device)
+        self.L = w.n_layers if n_layers is None else n_layers
+        self.n_rot = n_rot
+        self.parent, self.rank = tr.tr_template_from_branching(w.branching, w.n_nodes)
+        self.ctx = tr.tr_init(w.vocab, w.k, self.parent, self.rank, batch=w.batch, device=device)
+        B, N, V = w.batch, w.n_nodes, w.vocab
+        # --- integer loop state
+        self.M0 = np.zeros((B, V, w.k), dtype=np.int32) if zero_matrix else synth.seeded_matrix(w)
+        for b in range(B):
+            tr.tr_matrix_import(self.ctx, b, self.M0[b])
+        self.root0 = synth.root_tokens(w)
+        self.succ = synth.zipf_successors(w)
+        self.noise = synth.noise_logits(w, n_rot)                       # host copy for the checker's side
+        self.d_noise = torch.from_numpy(self.noise).to(self.dev)
+        self.d_logits = self.d_noise.clone()                           # [R, B, N, V], patched in place
+        self.d_prev_col = torch.full((n_rot, B, N), -1, dtype=torch.int32, device=self.dev)
+        self.d_succ = torch.from_numpy(self.succ).to(self.dev)
+        self.d_root = torch.from_numpy(self.root0).to(self.dev)
+        self.d_tree = torch.zeros(B, N, dtype=torch.int32, device=self.dev)
+        self.out_struct, self.out = tr.make_step_out(self.ctx)
+        self.out_struct.d_next_tree = self.d_tree.data_ptr()           # next tree replaces the current one
+        tr.tr_build_tree(self.ctx, self.d_root, self.d_tree)
+        # --- attention state
+        self.attn = None
+        if with_attention:
+            q, k, v = synth.attention_inputs(w, self.L)
+            self.q, self.k, self.v = (bf16_tensor(x, self.dev) for x in (q, k, v))
+            self.o = torch.zeros_like(self.q)
+            self.d_ctx_len = torch.tensor(list(w.ctx), dtype=torch.int32, device=self.dev)
+            self.attn = tr.make_attn_args(self.ctx, self.q, self.k, self.v, self.o, self.d_ctx_len, w.max_ctx,
+                                          splits=splits)
+        torch.cuda.synchronize(self.dev)
+
+    # one whole step: toy-model logits for the current tree, attention over all layers, verify/update/retrieve
+    def step(self, i, stream=None):
+        r = i % self.n_rot
+        tr.trs_patch_logits(self.d_logits[r], self.d_noise[r], self.d_tree, self.d_prev_col[r], self.d_succ,
+                            self.w.boost, stream)
+        if self.attn is not None:
+            tr.tr_tree_attention(self.ctx, self.attn, stream)
+        tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, stream)
+
+    def capture_graphs(self):
+        """One CUDA graph per rotating logits buffer; replay graphs[i % n_rot] for step i."""
+        graphs = []
+        s = torch.cuda.Stream(self.dev)
+        with torch.cuda.stream(s):
+            for r in range(self.n_rot):
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=s):
+                    self.step(r, stream=s)
+                graphs.append(g)
+        torch.cuda.synchronize(self.dev)
+        return graphs
+
+    def kernels_per_step(self):
+        n = 3  # logits patch (harness), top-k, accept/update/retrieve
+        if self.attn is not None:
+            n += 1
+            base = self.w.batch * self.L * self.w.n_q_heads
+            if self.attn.splits != 1 and base < 2 * 148:
+                n += 1  # split-KV combine
+        return n
+
+    def snapshot(self):
+        torch.cuda.synchronize(self.dev)
+        return {k: v.cpu().numpy().copy() for k, v in self.out.items()} | {"tree": self.d_tree.cpu().numpy().copy()}
+
+    def close(self):
+        tr.tr_destroy(self.ctx)

@@ -1,0 +1,296 @@
+"""GPU parity: every kernel, called through the C-ABI binding, against the CPU oracle on the same seeded inputs.
+Integer outputs are compared bit for bit; attention within max|diff| <= 2e-2 and relative L2 <= 1e-2."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import tr_oracle as orc
+from paper_2408_08696_b200 import synth
+from tests.oracle_loop import OracleLoop, attention_close, compare_step, oracle_attention
+
+pytestmark = pytest.mark.gpu
+
+ATOL, RTOL = 2e-2, 1e-2
+
+
+@pytest.fixture(scope="module")
+def tr():
+    from paper_2408_08696_b200 import build
+    build.build()
+    from paper_2408_08696_b200 import binding
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    return binding
+
+
+@pytest.fixture(scope="module")
+def harness(tr):
+    from paper_2408_08696_b200 import harness
+    return harness
+
+
+# ------------------------------------------------------------------ argmax + top-k
+def _topk_case(tr, logits, k, branching=(4, 2, 1), n=None):
+    rows, V = logits.shape
+    n = rows if n is None else n
+    parent, rank = tr.tr_template_from_branching(branching, n)
+    assert len(parent) == n
+    ctx = tr.tr_init(V, k, parent, rank, batch=rows // n)
+    out_struct, out = tr.make_step_out(ctx)
+    d_logits = torch.from_numpy(logits).cuda().reshape(rows // n, n, V)
+    d_tree = torch.zeros(rows // n, n, dtype=torch.int32, device="cuda")
+    tr.tr_verify_update(ctx, d_logits, d_tree, out_struct)
+    torch.cuda.synchronize()
+    got = out["topk_idx"].cpu().numpy().reshape(rows, k)
+    assert tr.tr_device_flags(ctx) == 0
+    tr.tr_destroy(ctx)
+    return got
+
+
+@pytest.mark.parametrize("V,k", [(1000, 8), (32000, 8), (33, 8), (4097, 8), (8191, 4), (12289, 16), (8, 8),
+                                 (50001, 1), (128256, 8)])
+def test_topk_matches_oracle_random(tr, V, k):
+    rng = np.random.default_rng(V * 31 + k)
+    x = rng.standard_normal((15, V)).astype(np.float32)
+    assert (_topk_case(tr, x, k) == orc.argtopk(x, k)).all()
+
+
+@pytest.mark.parametrize("V", [1000, 4099, 32000])
+def test_topk_ties_and_special_values(tr, V):
+    rng = np.random.default_rng(V)
+    x = rng.integers(-2, 3, size=(15, V)).astype(np.float32)          # five distinct values: ties everywhere
+    x[1] = 0.0
+    x[2] = -np.inf
+    x[3, ::2] = -0.0
+    x[3, 1::2] = 0.0
+    x[4] = np.float32(3.0)
+    x[4, V - 1] = np.float32(3.5)                                     # winner in the ragged last segment
+    x[5, : V // 2] = -np.inf
+    x[6] = np.arange(V, dtype=np.float32)                             # ascending: top-k at the very end
+    x[7] = -np.arange(V, dtype=np.float32)
+    x[8] = np.inf
+    x[9, :] = -1e30
+    x[9, 4096 % V] = 1e-30
+    assert (_topk_case(tr, x, 8) == orc.argtopk(x, 8)).all()
+
+
+def test_topk_adversarial_all_top_in_one_thread(tr):
+    # every one of a thread's 16 register slots beats the rest of the segment: the candidate buffer's bound
+    V = 8192
+    x = np.full((15, V), -5.0, dtype=np.float32)
+    for t in range(16):
+        x[:, 4 * 7 + (t // 4) * 1024 + t % 4] = 10.0 - t               # the 16 elements of thread 7, segment 0
+    x[:, 5000] = 9.5
+    assert (_topk_case(tr, x, 8) == orc.argtopk(x, 8)).all()
+
+
+# ------------------------------------------------------------------ retrieval
+def test_build_tree_matches_oracle(tr):
+    w = synth.WORKLOADS["llama2-70b-b8"]
+    parent, rank = tr.tr_template_from_branching(w.branching, w.n_nodes)
+    ctx = tr.tr_init(w.vocab, w.k, parent, rank, batch=w.batch)
+    M = synth.seeded_matrix(w)
+    for b in range(w.batch):
+        tr.tr_matrix_import(ctx, b, M[b])
+        assert (tr.tr_matrix_export(ctx, b) == M[b]).all()
+    roots = synth.root_tokens(w)
+    d_root = torch.from_numpy(roots).cuda()
+    d_tree = torch.zeros(w.batch, w.n_nodes, dtype=torch.int32, device="cuda")
+    tr.tr_build_tree(ctx, d_root, d_tree)
+    got = d_tree.cpu().numpy()
+    for b in range(w.batch):
+        assert (got[b] == orc.bfs_tree(M[b], parent, rank, int(roots[b]))).all()
+    # zero matrix (cold start, Sec. 3.1): all drafts are token 0
+    tr.tr_matrix_zero(ctx)
+    tr.tr_build_tree(ctx, d_root, d_tree)
+    got = d_tree.cpu().numpy()
+    assert (got[:, 0] == roots).all() and (got[:, 1:] == 0).all()
+    assert tr.tr_device_flags(ctx) == 0
+    # a root outside the vocabulary sets the flag and is treated as token 0; nothing traps
+    d_root[0] = w.vocab + 5
+    tr.tr_build_tree(ctx, d_root, d_tree)
+    assert tr.tr_device_flags(ctx) & tr.TR_FLAG_BAD_TOKEN
+    tr.tr_destroy(ctx)
+
+
+# ------------------------------------------------------------------ verify / update / retrieve loop
+def _run_loop(harness, w, steps, zero_matrix=False, graphs=False, check_every=1):
+    dw = harness.DeviceWorkload(w, with_attention=False, zero_matrix=zero_matrix)
+    ol = OracleLoop(w, zero_matrix=zero_matrix)
+    assert (dw.d_tree.cpu().numpy() == np.stack(ol.S)).all()
+    g = dw.capture_graphs() if graphs else None
+    mats = []
+    for i in range(steps):
+        if graphs:
+            g[i % dw.n_rot].replay()
+        else:
+            dw.step(i)
+        recs = ol.step(i)
+        if i % check_every == 0 or i == steps - 1:
+            compare_step(recs, dw.snapshot(), dw.ctx.max_new)
+        mats.append(np.mean([r["n_new"] for r in recs]))
+    from paper_2408_08696_b200 import binding as tr
+    for b in range(w.batch):
+        assert (tr.tr_matrix_export(dw.ctx, b) == ol.M[b]).all(), "matrix differs after the loop"
+    assert tr.tr_device_flags(dw.ctx) == 0
+    dw.close()
+    return float(np.mean(mats))
+
+
+def test_loop_tiny_50_steps(harness):
+    mat = _run_loop(harness, synth.WORKLOADS["tiny"], 50)
+    assert 1.0 <= mat <= 7.0
+
+
+def test_loop_tiny_cold_start_zero_matrix(harness):
+    _run_loop(harness, synth.WORKLOADS["tiny"], 30, zero_matrix=True)     # all-equal drafts: duplicate handling
+
+
+def test_loop_llama2_7b_shape(harness):
+    _run_loop(harness, synth.WORKLOADS["llama2-7b"], 24)
+
+
+def test_loop_batched_8_sequences_via_graph(harness):
+    _run_loop(harness, synth.WORKLOADS["llama2-70b-b8"], 12, graphs=True)
+
+
+def test_loop_large_vocab(harness):
+    _run_loop(harness, synth.WORKLOADS["llama3-8b"], 6)
+
+
+def test_duplicate_tokens_last_writer_wins(tr):
+    # Appendix "Explanation of Three Update Strategies": S = [a, b, c, a, d] keeps O[3] for a.
+    parent = np.array([-1, 0, 0, 0, 0], dtype=np.int32)
+    rank = np.array([0, 0, 1, 2, 3], dtype=np.int32)
+    V, k = 64, 4
+    ctx = tr.tr_init(V, k, parent, rank)
+    out_struct, out = tr.make_step_out(ctx)
+    S = np.array([[10, 11, 12, 10, 13]], dtype=np.int32)
+    rng = np.random.default_rng(0)
+    logits = rng.standard_normal((1, 5, V)).astype(np.float32)
+    d_tree = torch.from_numpy(S).cuda()
+    tr.tr_verify_update(ctx, torch.from_numpy(logits).cuda(), d_tree, out_struct)
+    torch.cuda.synchronize()
+    M = tr.tr_matrix_export(ctx, 0)
+    O = orc.argtopk(logits[0], k)
+    assert (M[10] == O[3]).all() and not (M[10] == O[0]).all()
+    assert (M[11] == O[1]).all() and (M[12] == O[2]).all() and (M[13] == O[4]).all()
+    touched = np.zeros(V, bool); touched[[10, 11, 12, 13]] = True
+    assert (M[~touched] == 0).all()
+    tr.tr_destroy(ctx)
+
+
+# ------------------------------------------------------------------ tree attention
+def _attention_case(harness, w, n_layers, splits=0):
+    dw = harness.DeviceWorkload(w, n_layers=n_layers, splits=splits)
+    from paper_2408_08696_b200 import binding as tr
+    tr.tr_tree_attention(dw.ctx, dw.attn)
+    torch.cuda.synchronize()
+    got = dw.o.float().cpu().numpy()                                   # [B, L, N, Hq, D]
+    q, k, v = synth.attention_inputs(w, n_layers)
+    worst = (0.0, 0.0)
+    for b in range(w.batch):
+        for l in range(n_layers):
+            ref = oracle_attention(w, q, k, v, b, l, dw.parent)
+            assert np.isfinite(got[b, l]).all()
+            for h in range(w.n_q_heads):
+                mx, rel = attention_close(got[b, l, :, h], ref[:, h])
+                assert mx <= ATOL and rel <= RTOL, (b, l, h, mx, rel)
+                worst = (max(worst[0], mx), max(worst[1], rel))
+    dw.close()
+    return worst
+
+
+@pytest.mark.parametrize("splits", [0, 1, 2, 3, 5])
+def test_attention_tiny(harness, splits):
+    _attention_case(harness, synth.WORKLOADS["tiny"], 1, splits)
+
+
+@pytest.mark.parametrize("ctx", [0, 1, 63, 64, 65, 77, 200])
+def test_attention_ragged_context(harness, ctx):
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], ctx=(ctx,))
+    _attention_case(harness, w, 2)
+    _attention_case(harness, w, 1, splits=4)
+
+
+@pytest.mark.parametrize("splits", [0, 1, 4])
+def test_attention_head_dim_128_full_tree(harness, splits):
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=4, n_kv_heads=4, ctx=(333,))
+    _attention_case(harness, w, 2, splits)
+
+
+def test_attention_gqa_and_batch_with_mixed_contexts(harness):
+    w = dataclasses.replace(synth.WORKLOADS["llama2-70b-b8"], n_q_heads=8, n_kv_heads=2, ctx=(100, 257, 31))
+    _attention_case(harness, w, 2)
+    _attention_case(harness, w, 1, splits=3)
+
+
+def test_attention_single_node_tree(harness):
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], n_nodes=1, branching=(1,), ctx=(50,))
+    _attention_case(harness, w, 1)
+
+
+def test_attention_llama2_7b_full_size_sampled(harness):
+    """The benchmark's launch configuration (32 layers x 32 heads in one launch, 1024-token prefix); the oracle
+    checks a seeded sample of (layer, head) outputs."""
+    w = synth.WORKLOADS["llama2-7b"]
+    dw = harness.DeviceWorkload(w)
+    from paper_2408_08696_b200 import binding as tr
+    tr.tr_tree_attention(dw.ctx, dw.attn)
+    torch.cuda.synchronize()
+    pool = synth.normal_pool(w.seed)
+    rng = np.random.default_rng(123)
+    for _ in range(24):
+        l, h = int(rng.integers(0, w.n_layers)), int(rng.integers(0, w.n_q_heads))
+        qs, ks, vs = synth.attention_slice(w, pool, 0, l, h)
+        ref = orc.tree_attention(synth.bf16_bits_to_f32(qs[:, h:h + 1]), synth.bf16_bits_to_f32(ks)[None],
+                                 synth.bf16_bits_to_f32(vs)[None], w.ctx[0], dw.parent)
+        got = dw.o[0, l, :, h].float().cpu().numpy()
+        mx, rel = attention_close(got, ref[:, 0])
+        assert mx <= ATOL and rel <= RTOL, (l, h, mx, rel)
+    assert torch.isfinite(dw.o.float()).all()
+    dw.close()
+
+
+# ------------------------------------------------------------------ whole step, host-buffer entry point
+def test_step_host_matches_device_calls(harness, tr):
+    import ctypes as C
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], ctx=(100,))
+    L = 2
+    dw = harness.DeviceWorkload(w, n_layers=L)
+    ol = OracleLoop(w)
+    B, N, V, Hq, Hkv, D = w.batch, w.n_nodes, w.vocab, w.n_q_heads, w.n_kv_heads, w.head_dim
+    q, k, v = synth.attention_inputs(w, L)
+    c = w.ctx[0]
+    h_q = torch.from_numpy(q.view(np.int16)).pin_memory()
+    h_tk = torch.from_numpy(np.ascontiguousarray(k[:, :, :, c:c + N]).view(np.int16)).pin_memory()
+    h_tv = torch.from_numpy(np.ascontiguousarray(v[:, :, :, c:c + N]).view(np.int16)).pin_memory()
+    dw.k[:, :, :, c:c + N] = 0          # the call itself must place the tree rows
+    dw.v[:, :, :, c:c + N] = 0
+    logits = np.stack([synth.step_logits(ol.noise[0, b], ol.S[b], ol.succ, w.boost) for b in range(B)])
+    h_logits = torch.from_numpy(logits).pin_memory()
+    h_ctx = np.array(w.ctx, dtype=np.int32)
+    h_out = torch.zeros(B, L, N, Hq, D, dtype=torch.bfloat16).pin_memory()
+    h_n_new = torch.zeros(B, dtype=torch.int32).pin_memory()
+    h_tokens = torch.zeros(B, dw.ctx.max_new, dtype=torch.int32).pin_memory()
+    h_next = torch.zeros(B, N, dtype=torch.int32).pin_memory()
+    io = tr.tr_host_io()
+    io.h_q, io.h_tree_k, io.h_tree_v = h_q.data_ptr(), h_tk.data_ptr(), h_tv.data_ptr()
+    io.h_logits, io.h_ctx_len = h_logits.data_ptr(), h_ctx.ctypes.data
+    io.d_logits_staging, io.d_tree = dw.d_logits[0].data_ptr(), dw.d_tree.data_ptr()
+    io.h_out, io.h_n_new, io.h_out_tokens, io.h_next_tree = (h_out.data_ptr(), h_n_new.data_ptr(),
+                                                             h_tokens.data_ptr(), h_next.data_ptr())
+    dw.q.zero_()
+    tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)
+    recs = ol.step(0)
+    compare_step(recs, dw.snapshot(), dw.ctx.max_new)
+    assert h_n_new[0].item() == recs[0]["n_new"]
+    assert h_tokens[0, : recs[0]["n_new"]].tolist() == recs[0]["out_tokens"]
+    assert (h_next[0].numpy() == recs[0]["next_tree"]).all()
+    for l in range(L):
+        ref = oracle_attention(w, q, k, v, 0, l, dw.parent)
+        for h in range(Hq):
+            mx, rel = attention_close(h_out[0, l, :, h].float().numpy(), ref[:, h])
+            assert mx <= ATOL and rel <= RTOL
+    dw.close()
