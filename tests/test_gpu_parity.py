@@ -31,7 +31,7 @@ def harness(tr):
 
 
 # ------------------------------------------------------------------ argmax + top-k
-def _topk_case(tr, logits, k, branching=(4, 2, 1), n=None):
+def _topk_case(tr, logits, k, branching=(1,), n=None):
     rows, V = logits.shape
     n = rows if n is None else n
     parent, rank = tr.tr_template_from_branching(branching, n)
