@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the Token Recycling verify-and-recycle step on B200.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload llama2-7b]
+
+One step = toy-model logits patch (harness) -> tree attention over all layers (one launch) -> fused
+argmax/top-k -> accept + matrix update + next-tree retrieval, replayed as one CUDA graph per step with all
+state resident on the device.  Prints ONE JSON line (rank 0).  With N > 1 every rank runs an independent
+replica on its own GPU (the step has no exchange between GPUs); the job's time is the slowest rank's.
+`--impl reference` times the CPU oracle (the checker the tests use) on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "us per TR verify-and-recycle step"
+UNIT = "us/step"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+def algorithmic_bytes(w, n_layers):
+    """Bytes the method must move per step: K/V once, Q and O once, logits once, 2N matrix rows."""
+    N, D = w.n_nodes, w.head_dim
+    kv = sum(2 * w.n_kv_heads * (c + N) * D * 2 for c in w.ctx) * n_layers
+    qo = 2 * w.batch * N * w.n_q_heads * D * 2 * n_layers
+    logits = w.batch * N * w.vocab * 4
+    matrix = w.batch * 2 * N * w.k * 4 + w.batch * N * w.k * 4       # rows written + rows gathered + top-k out
+    return {"attention": kv + qo, "logits": logits, "matrix": matrix, "total": kv + qo + logits + matrix}
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 6:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------------
+class OracleSampler:
+    """Times the CPU oracle, as it stands, on a bounded sample of one step of workload `w`: `n_units` of the
+    (sequence, layer, kv-head) attention units, scaled to all of them, plus one full top-k / accept / update /
+    retrieve pass per sequence."""
+
+    def __init__(self, w):
+        from oracle import tr_oracle as orc
+        from paper_2408_08696_b200 import synth
+        self.orc, self.synth, self.w = orc, synth, w
+        try:
+            from threadpoolctl import threadpool_info
+            self.threads = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+        except Exception:
+            self.threads = 1
+        self.parent, self.rank = orc.template_from_branching(w.branching, w.n_nodes)
+        self.pool = synth.normal_pool(w.seed)
+        self.rng = np.random.default_rng(7)
+        self.units_total = w.batch * w.n_layers * w.n_kv_heads
+        self.M = synth.seeded_matrix(w)[0].astype(np.int64)
+        self.succ = synth.zipf_successors(w)
+        self.noise = synth.noise_logits(w, 1)[0]
+        self.S = orc.bfs_tree(self.M, self.parent, self.rank, int(synth.root_tokens(w)[0]))
+
+    def step_us(self, n_units):
+        w, orc, synth = self.w, self.orc, self.synth
+        group = w.n_q_heads // w.n_kv_heads
+        n_units = min(n_units, self.units_total)
+        t_attn = 0.0
+        for _ in range(n_units):
+            b = int(self.rng.integers(0, w.batch))
+            l, g = int(self.rng.integers(0, w.n_layers)), int(self.rng.integers(0, w.n_kv_heads))
+            qs, ks, vs = synth.attention_slice(w, self.pool, b, l, g)
+            qf = synth.bf16_bits_to_f32(qs[:, g * group:(g + 1) * group])
+            kf, vf = synth.bf16_bits_to_f32(ks)[None], synth.bf16_bits_to_f32(vs)[None]
+            t0 = time.perf_counter()
+            orc.tree_attention(qf, kf, vf, w.ctx[b], self.parent)
+            t_attn += time.perf_counter() - t0
+        logits = synth.step_logits(self.noise[0], self.S, self.succ, w.boost)
+        t0 = time.perf_counter()
+        rec = orc.verify_update(self.M, self.S, logits, self.parent, self.rank)
+        t_int = (time.perf_counter() - t0) * w.batch
+        self.S = rec["next_tree"]
+        return (t_attn / n_units * self.units_total + t_int) * 1e6
+
+    def describe(self, n_units, steps):
+        return ("%d step(s); per step %d of %d (sequence, layer, kv-head) attention units timed and scaled to all, "
+                "plus one full top-k/accept/update/retrieve pass per sequence"
+                % (steps, min(n_units, self.units_total), self.units_total))
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: K steps, each a bounded sample scaled to a whole step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSampler(w)
+    n_units = 32
+    vals = [smp.step_us(n_units) for _ in range(args.warmup + args.steps)][args.warmup:]
+    v = float(np.mean(vals))
+    line = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": v / 1000.0, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": w.name, "note": "CPU oracle on host cores; each step is a bounded sample scaled up"},
+        "cpu_baseline": {"value": v, "unit": UNIT, "cores": smp.threads, "kind": "oracle",
+                         "sample": smp.describe(n_units, args.steps)},
+        "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_2408_08696_b200 import binding as tr
+    from paper_2408_08696_b200 import harness, replicas, synth
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the step has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    K, W = args.steps, max(args.warmup, 3)
+
+    dw = harness.DeviceWorkload(w, n_layers=args.layers or None, device=local_rank)
+    graphs = dw.capture_graphs()
+    if args.profile:
+        for i in range(W + K):
+            graphs[i % dw.n_rot].replay()
+        torch.cuda.synchronize()
+        dw.close()
+        return
+    stream = torch.cuda.current_stream()
+    for i in range(W):
+        graphs[i % dw.n_rot].replay()
+    torch.cuda.synchronize()
+
+    # ---- timed region: K graph replays back to back, device time between two events on the launching stream
+    replicas.barrier()
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_new_sum = 0
+    e0.record(stream)
+    for i in range(K):
+        graphs[(W + i) % dw.n_rot].replay()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    replicas.barrier()
+    elapsed_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if sampler else None
+    agg = replicas.aggregate(elapsed_ms, K, device=dev if world > 1 else "cpu")
+    n_new_sum = int(dw.out["n_new"].sum().item())
+    flags = tr.tr_device_flags(dw.ctx)
+
+    # ---- dominant kernel (tree attention) alone: event pair around every launch, same stream
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for i in range(K):
+        tr.trs_patch_logits(dw.d_logits[i % dw.n_rot], dw.d_noise[i % dw.n_rot], dw.d_tree,
+                            dw.d_prev_col[i % dw.n_rot], dw.d_succ, w.boost)
+        ev[i][0].record(stream)
+        tr.tr_tree_attention(dw.ctx, dw.attn)
+        ev[i][1].record(stream)
+        tr.tr_verify_update(dw.ctx, dw.d_logits[i % dw.n_rot], dw.d_tree, dw.out_struct)
+    torch.cuda.synchronize()
+    attn_ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
+    # per-layer launches (one call per layer, as a real model's forward would issue them), for the record
+    per_layer_ms = None
+    if dw.L > 1:
+        qs = [dw.q[:, l:l + 1] for l in range(dw.L)]
+        args_l = [tr.make_attn_args(dw.ctx, dw.q[:, l:l + 1], dw.k[:, l:l + 1], dw.v[:, l:l + 1], dw.o[:, l:l + 1],
+                                    dw.d_ctx_len, w.max_ctx) for l in range(dw.L)]
+        gl = torch.cuda.CUDAGraph()
+        s2 = torch.cuda.Stream(dev)
+        with torch.cuda.stream(s2):
+            with torch.cuda.graph(gl, stream=s2):
+                for a in args_l:
+                    tr.tr_tree_attention(dw.ctx, a, s2)
+        torch.cuda.synchronize()
+        for _ in range(3):
+            gl.replay()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for _ in range(20):
+            gl.replay()
+        a1.record(stream)
+        torch.cuda.synchronize()
+        per_layer_ms = a0.elapsed_time(a1) / 20
+
+    # ---- end to end through the host-buffer entry point: pinned inputs in, results out, every step
+    B, N, V, Hq, Hkv, D, L = w.batch, w.n_nodes, w.vocab, w.n_q_heads, w.n_kv_heads, w.head_dim, dw.L
+    h_q = dw.q.cpu().pin_memory()
+    h_tk = torch.stack([dw.k[b, :, :, c:c + N] for b, c in enumerate(w.ctx)]).cpu().contiguous().pin_memory()
+    h_tv = torch.stack([dw.v[b, :, :, c:c + N] for b, c in enumerate(w.ctx)]).cpu().contiguous().pin_memory()
+    h_logits = [dw.d_noise[r].cpu().pin_memory() for r in range(dw.n_rot)]
+    h_ctx = np.array(w.ctx, dtype=np.int32)
+    h_out = torch.zeros(B, L, N, Hq, D, dtype=torch.bfloat16).pin_memory()
+    h_n_new = torch.zeros(B, dtype=torch.int32).pin_memory()
+    h_tok = torch.zeros(B, dw.ctx.max_new, dtype=torch.int32).pin_memory()
+    h_next = torch.zeros(B, N, dtype=torch.int32).pin_memory()
+    d_stage = torch.empty(B, N, V, dtype=torch.float32, device=dev)
+    io = tr.tr_host_io()
+    io.h_q, io.h_tree_k, io.h_tree_v = h_q.data_ptr(), h_tk.data_ptr(), h_tv.data_ptr()
+    io.h_ctx_len, io.d_logits_staging, io.d_tree = h_ctx.ctypes.data, d_stage.data_ptr(), dw.d_tree.data_ptr()
+    io.h_out, io.h_n_new, io.h_out_tokens, io.h_next_tree = (h_out.data_ptr(), h_n_new.data_ptr(), h_tok.data_ptr(),
+                                                             h_next.data_ptr())
+    h2d = h_q.numel() * 2 + h_tk.numel() * 2 + h_tv.numel() * 2 + h_logits[0].numel() * 4
+    d2h = h_out.numel() * 2 + h_n_new.numel() * 4 + h_tok.numel() * 4 + h_next.numel() * 4
+    Ke = max(3, min(K, 20))
+    for i in range(2):
+        io.h_logits = h_logits[i % dw.n_rot].data_ptr()
+        tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)
+    replicas.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for i in range(Ke):
+        io.h_logits = h_logits[i % dw.n_rot].data_ptr()
+        tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)      # synchronises the stream itself
+    e2e_ms = (time.perf_counter() - t0) * 1000.0
+    e2e = replicas.aggregate(e2e_ms, Ke, device=dev if world > 1 else "cpu")
+
+    if rank == 0:
+        peak, peak_src = load_peaks()
+        ab = algorithmic_bytes(w, dw.L)
+        attn_gbs = ab["attention"] / (attn_ms * 1e-3) / 1e9
+        step_gbs = ab["total"] / (agg["ms_per_step"] * 1e-3) / 1e9
+        smp = OracleSampler(w)
+        cpu_units, cpu_steps = 2048, 3                       # roughly 15-20 s of host work at the 7B shape
+        cpu_us = float(np.mean([smp.step_us(cpu_units) for _ in range(cpu_steps)]))
+        cpu_desc, cpu_threads = smp.describe(cpu_units, cpu_steps), smp.threads
+        line = {
+            "metric": METRIC, "value": agg["us_per_step_job"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+            "ms_per_step": agg["ms_per_step"], "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": w.name, "vocab": V, "k": w.k, "tree_nodes": N, "layers": L, "q_heads": Hq,
+                       "kv_heads": Hkv, "head_dim": D, "context": list(w.ctx), "batch": B,
+                       "attention_launch": "all layers in one launch",
+                       "l2": "inputs larger than L2: %.0f MB of K/V streamed per step" % (ab["attention"] / 1e6),
+                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+            "steps_per_s": agg["steps_per_s"],
+            "step_hbm": {"algorithmic_bytes": ab["total"], "achieved_gbs": step_gbs, "frac_of_measured": step_gbs / peak,
+                         "frac_of_8tbs": step_gbs / 8000.0},
+            "roofline": {"kernel": "tree attention (all layers)", "bound": "hbm", "achieved": attn_gbs, "peak": peak,
+                         "unit": "GB/s", "frac": attn_gbs / peak, "peak_source": peak_src,
+                         "algorithmic_bytes_per_launch": ab["attention"], "avg_launch_ms": attn_ms,
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+            "attention_per_layer_launches_ms": per_layer_ms,
+            "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},
+            "e2e": {"value": e2e["us_per_step_job"], "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                    "steps": Ke},
+            "gpu_launches": dw.kernels_per_step() * K,
+            "clocks": clocks,
+            "new_tokens_last_step": n_new_sum / B,
+            "device_flags": flags,
+        }
+        print(json.dumps(line), flush=True)
+    dw.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# DRAM bytes (read + write) of one attention launch from the committed ncu capture (see profiles/), per workload.
+NCU_TRAFFIC_BYTES = {}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama2-7b")
+    ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
+    ap.add_argument("--profile", action="store_true",
+                    help="only warm up and replay the step graph K times (for ncu); prints no bench line")
+    args = ap.parse_args()
+    from paper_2408_08696_b200 import synth
+    w = synth.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()
