@@ -318,7 +318,17 @@ tr_status tr_attention_mma_setup() {
   return TR_OK;
 }
 
-tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s) {
+static AttnParams make_params(tr_ctx* ctx, const tr_attn_args* a);
+
+// Split-KV merge for either attention kernel (both write the same partial format).
+void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s) {
+  AttnParams p = make_params(ctx, a);
+  p.S = S;
+  const unsigned base = static_cast<unsigned>(ctx->batch) * a->n_layers * a->n_q_heads;
+  tr_attn_combine_kernel<<<dim3(ctx->n_nodes, base), a->head_dim, 0, s>>>(p, a->head_dim);
+}
+
+static AttnParams make_params(tr_ctx* ctx, const tr_attn_args* a) {
   AttnParams p;
   p.q = static_cast<const __nv_bfloat16*>(a->q);
   p.k = static_cast<const __nv_bfloat16*>(a->k_cache);
@@ -334,6 +344,12 @@ tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream
   p.os_b = a->o_stride[0]; p.os_h = a->o_stride[1]; p.os_t = a->o_stride[2]; p.os_l = a->layer_stride_o;
   const float scale = a->scale != 0.f ? a->scale : 1.0f / sqrtf(static_cast<float>(a->head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
+  p.S = 1;
+  return p;
+}
+
+tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s) {
+  AttnParams p = make_params(ctx, a);
   const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * a->n_q_heads;
   if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
   p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BN);
@@ -348,7 +364,7 @@ tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream
     tr_attn_mma_kernel<64><<<grid, nwarps * 32, smem, s>>>(p);
   TR_CUDA_TRY(cudaGetLastError());
   if (p.S > 1) {
-    tr_attn_combine_kernel<<<dim3(ctx->n_nodes, static_cast<unsigned>(base)), D, 0, s>>>(p, D);
+    tr_launch_attention_combine(ctx, a, p.S, s);
     TR_CUDA_TRY(cudaGetLastError());
   }
   return TR_OK;

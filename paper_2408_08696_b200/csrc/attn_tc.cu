@@ -1,0 +1,584 @@
+// Tree attention (paper Sec. 2.2) for head_dim 128 on the 5th-generation tensor cores: a persistent,
+// warp-specialised flash-decoding kernel.
+//
+//   warp 0      TMA producer: Q tile (double-buffered) and a ring of 32 KB K / V tiles (128 keys x 128 dims, bf16,
+//               128-byte swizzle), one mbarrier per ring slot
+//   warp 1      MMA issuer: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM) and
+//               O += P V (P read from TMEM, V as an MN-major shared-memory operand); owns the TMEM allocation
+//   warps 2..5  softmax: thread r owns query row r (= TMEM lane r): loads its S row, applies the ancestor mask
+//               (a 128-bit mask kept in registers, shifted to the tile), exp2 with a lazily updated reference
+//               maximum, writes P (bf16) over S in TMEM, rescales O in TMEM only when the maximum moved by
+//               more than 2^8, and finally normalises and stores the output row
+//
+// A CTA walks units u = blockIdx.x, blockIdx.x + gridDim.x, ...; a unit is one (sequence, layer, KV head,
+// query head, KV split).  TMEM: S/P double buffer (2 x 128 columns) + O double buffer (2 x 128 columns), so the
+// QK^T of tile j+1 overlaps the softmax of tile j and the epilogue of a unit overlaps the next unit.
+// Every wait is bounded; a wait that runs out sets TR_FLAG_WAIT_TIMEOUT and the CTA drains and exits.
+#include <cuda.h>
+
+#include "tr_internal.cuh"
+
+namespace {
+
+constexpr int BK = 128;          // keys per tile
+constexpr int HD = 128;          // head_dim
+constexpr int NST = 5;           // ring slots (K and V tiles alternate)
+constexpr int TILE_BYTES = BK * HD * 2;       // 32 KB
+constexpr int HALF_BYTES = TILE_BYTES / 2;    // one TMA box: 64 dims x 128 rows
+constexpr int NTHREADS = 192;
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about two seconds of SM clock
+
+struct TcParams {
+  __nv_bfloat16* out;
+  const int32_t* ctx_len;
+  const uint32_t* anc;
+  float* part_o;
+  float* part_ml;
+  uint32_t* flags;
+  int N, Hq, Hkv, L, S, n_units;
+  int64_t os_b, os_h, os_t, os_l;
+  float scale_log2;
+};
+
+// shared memory map (offsets from a 1024-byte aligned base)
+constexpr int SM_Q = 0;                               // 2 x 32 KB
+constexpr int SM_RING = 2 * TILE_BYTES;               // NST x 32 KB
+constexpr int SM_BAR = SM_RING + NST * TILE_BYTES;    // mbarriers
+constexpr int BAR_FULL = 0, BAR_EMPTY = NST, BAR_QFULL = 2 * NST, BAR_QEMPTY = BAR_QFULL + 2,
+              BAR_SFULL = BAR_QEMPTY + 2, BAR_PFULL = BAR_SFULL + 2, BAR_PVDONE = BAR_PFULL + 2,
+              BAR_OFREE = BAR_PVDONE + 2, BAR_COUNT = BAR_OFREE + 2;
+constexpr int SM_MISC = SM_BAR + BAR_COUNT * 8;       // tmem base (4 B), abort flag (4 B)
+constexpr int SM_TOTAL = SM_MISC + 16;
+constexpr int SMEM_BYTES = SM_TOTAL + 1024;           // slack for manual 1024-byte alignment
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n.reg .pred p;\n"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+      "selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok;
+}
+// Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completes.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (uint32_t i = 1;; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 0u) {
+      if (*abort_flag) return false;
+      if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
+    }
+  }
+  *abort_flag = 1u;
+  return false;
+}
+
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3, int c4) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, "
+      "%6, %7}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+      : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\n"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+      "%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
+      "%30,%31,%32};"
+      ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+        "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+        "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  `lbo`/`sbo` in bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+  uint64_t d = 0;
+  d |= static_cast<uint64_t>((addr >> 4) & 0x3FFFu);
+  d |= static_cast<uint64_t>((lbo >> 4) & 0x3FFFu) << 16;
+  d |= static_cast<uint64_t>((sbo >> 4) & 0x3FFFu) << 32;
+  d |= 1ull << 46;  // descriptor version for sm_100
+  d |= 2ull << 61;  // SWIZZLE_128B
+  return d;
+}
+// Instruction descriptor for kind::f16: bf16 x bf16 -> f32, M = 128, N = 128.
+__host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((b_mn_major ? 1u : 0u) << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+}
+
+struct Unit {
+  int b, layer, kvh, h, split, slot;
+  int t0, t1, C;
+};
+
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, int u) {
+  Unit x;
+  x.slot = u;
+  const int group = p.Hq / p.Hkv;
+  const int gq = u % group; u /= group;
+  x.split = u % p.S; u /= p.S;
+  x.kvh = u % p.Hkv; u /= p.Hkv;
+  x.layer = u % p.L; u /= p.L;
+  x.b = u;
+  x.h = x.kvh * group + gq;
+  x.C = p.ctx_len[x.b];
+  const int T = (x.C + p.N + BK - 1) / BK;
+  x.t0 = static_cast<int>(static_cast<int64_t>(T) * x.split / p.S);
+  x.t1 = static_cast<int>(static_cast<int64_t>(T) * (x.split + 1) / p.S);
+  return x;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                  const __grid_constant__ CUtensorMap map_v, const TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  const uint32_t raw = smem_u32(smem_raw);
+  const uint32_t base = (raw + 1023u) & ~1023u;
+  unsigned char* base_ptr = smem_raw + (base - raw);
+  const uint32_t bars = base + SM_BAR;
+  volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(base_ptr + SM_MISC);
+  volatile uint32_t* s_abort = s_tmem + 1;
+  auto bar = [&](int i) { return bars + static_cast<uint32_t>(i) * 8u; };
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+
+  if (tid == 0) {
+    for (int i = 0; i < NST; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(bar(BAR_QFULL + i), 1);
+      mbar_init(bar(BAR_QEMPTY + i), 1);
+      mbar_init(bar(BAR_SFULL + i), 1);
+      mbar_init(bar(BAR_PFULL + i), 128);
+      mbar_init(bar(BAR_PVDONE + i), 1);
+      mbar_init(bar(BAR_OFREE + i), 128);
+    }
+    *s_abort = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + SM_MISC), "r"(512u)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem = *s_tmem;
+
+  if (warp == 0) {
+    // =========================== TMA producer ===========================
+    if (lane == 0) {
+      uint32_t ui = 0, c = 0;  // non-empty units done by this CTA; ring entries issued
+      bool ok = true;
+      for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+        const Unit x = decode_unit(p, u);
+        if (x.t0 >= x.t1) continue;
+        const uint32_t qb = ui & 1u;
+        ok = mbar_wait(bar(BAR_QEMPTY + qb), ((ui >> 1) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        mbar_expect_tx(bar(BAR_QFULL + qb), TILE_BYTES);
+        tma_load_5d(base + SM_Q + qb * TILE_BYTES, &map_q, bar(BAR_QFULL + qb), 0, x.h, 0, x.layer, x.b);
+        tma_load_5d(base + SM_Q + qb * TILE_BYTES + HALF_BYTES, &map_q, bar(BAR_QFULL + qb), 64, x.h, 0, x.layer, x.b);
+        for (int t = x.t0; t < x.t1 && ok; ++t) {
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv) {
+            const uint32_t slot = c % NST, par = ((c / NST) & 1u) ^ 1u;
+            ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort);
+            if (!ok) break;
+            const CUtensorMap* m = kv == 0 ? &map_k : &map_v;
+            const uint32_t dst = base + SM_RING + slot * TILE_BYTES;
+            mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
+            tma_load_5d(dst, m, bar(BAR_FULL + slot), 0, t * BK, x.kvh, x.layer, x.b);
+            tma_load_5d(dst + HALF_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b);
+            ++c;
+          }
+        }
+        ++ui;
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // =========================== MMA issuer ===========================
+    if (lane == 0) {
+      constexpr uint32_t IDESC_QK = make_idesc(false);
+      constexpr uint32_t IDESC_PV = make_idesc(true);
+      uint32_t ui = 0, c = 0, g = 0;  // units, ring entries consumed, tiles (S buffers) issued
+      bool ok = true;
+      // software pipeline over tiles: QK(j+1) is issued before PV(j)
+      auto issue_qk = [&](uint32_t qb, uint32_t gg) -> bool {
+        const uint32_t sb = gg & 1u;
+        // the S/P buffer is free once PV of tile gg-2 has completed
+        if (!mbar_wait(bar(BAR_PVDONE + sb), ((gg >> 1) & 1u) ^ 1u, s_abort)) return false;
+        const uint32_t slot = c % NST;
+        if (!mbar_wait(bar(BAR_FULL + slot), (c / NST) & 1u, s_abort)) return false;
+        tc_fence_after();
+        const uint32_t qa = base + SM_Q + qb * TILE_BYTES, ka = base + SM_RING + slot * TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < HD / 16; ++k) {
+          const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
+          tc_mma_ss(tmem + sb * 128u, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK, k > 0);
+        }
+        tc_commit(bar(BAR_EMPTY + slot));   // K tile consumed
+        tc_commit(bar(BAR_SFULL + sb));     // S ready for the softmax warps
+        ++c;
+        return true;
+      };
+      for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+        const Unit x = decode_unit(p, u);
+        const int nt = x.t1 - x.t0;
+        if (nt <= 0) continue;
+        const uint32_t qb = ui & 1u, ob = ui & 1u;
+        ok = mbar_wait(bar(BAR_QFULL + qb), (ui >> 1) & 1u, s_abort);
+        if (!ok) break;
+        ok = issue_qk(qb, g);
+        for (int j = 0; j < nt && ok; ++j) {
+          // ring order is K0 V0 K1 V1 ...: V(j) sits at entry c, K(j+1) at entry c+1; the QK of tile j+1 goes
+          // first so that it overlaps the softmax of tile j
+          const uint32_t vslot = c % NST, vpar = (c / NST) & 1u;
+          ++c;
+          if (j + 1 < nt) {
+            ok = issue_qk(qb, g + 1);
+            if (!ok) break;
+          } else {
+            tc_commit(bar(BAR_QEMPTY + qb));  // all QK of this unit issued: Q buffer free when they finish
+          }
+          if (j == 0) {  // the O buffer must have been drained by the epilogue of unit ui-2
+            ok = mbar_wait(bar(BAR_OFREE + ob), ((ui >> 1) & 1u) ^ 1u, s_abort);
+            if (!ok) break;
+          }
+          const uint32_t sb = g & 1u;
+          ok = mbar_wait(bar(BAR_PFULL + sb), (g >> 1) & 1u, s_abort) && mbar_wait(bar(BAR_FULL + vslot), vpar, s_abort);
+          if (!ok) break;
+          tc_fence_after();
+          const uint32_t va = base + SM_RING + vslot * TILE_BYTES;
+#pragma unroll
+          for (int k = 0; k < BK / 16; ++k) {
+            // A = P (bf16 pairs, 8 TMEM columns per 16 keys); B = V tile, MN-major: 64-dim chunks 16 KB apart,
+            // 8-key groups 1 KB apart, 16 keys per step = 2 KB
+            tc_mma_ts(tmem + 256u + ob * 128u, tmem + sb * 128u + k * 8u, smem_desc(va + k * 2048, HALF_BYTES, 1024),
+                      IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
+          }
+          tc_commit(bar(BAR_EMPTY + vslot));  // V tile consumed
+          tc_commit(bar(BAR_PVDONE + sb));    // P consumed, O updated
+          ++g;
+        }
+        ++ui;
+      }
+    }
+    __syncwarp();
+  } else {
+    // =========================== softmax / correction / epilogue ===========================
+    const int r = (warp & 3) * 32 + lane;                 // query row == TMEM lane
+    const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
+    uint32_t anc[4];
+#pragma unroll
+    for (int w = 0; w < 4; ++w) anc[w] = r < p.N ? p.anc[r * 4 + w] : 0u;
+    uint32_t ui = 0, g = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+      const Unit x = decode_unit(p, u);
+      const int nt = x.t1 - x.t0;
+      float m_ref = -INFINITY, l = 0.f;
+      const uint32_t ob = ui & 1u;
+      for (int j = 0; j < nt && ok; ++j, ++g) {
+        const uint32_t sb = g & 1u;
+        ok = mbar_wait(bar(BAR_SFULL + sb), (g >> 1) & 1u, s_abort);
+        ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
+        if (!ok) break;
+        tc_fence_after();
+        uint32_t sreg[4][32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) tc_ld32(tmem + lane_base + sb * 128u + q * 32u, sreg[q]);
+        tc_wait_ld();
+        // visibility of the tile's 128 keys for this row
+        const int key0 = (x.t0 + j) * BK;
+        uint32_t vis[4] = {0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu, 0xFFFFFFFFu};
+        const bool masked = key0 + BK > x.C;
+        if (masked) {
+          const int s = x.C - key0;  // tile column of the first tree key (may be <= 0 or >= 128)
+#pragma unroll
+          for (int w = 0; w < 4; ++w) {
+            // bit c of word w: column 32w + c; visible iff column < s, or bit (column - s) of anc
+            uint32_t word = 0;
+            const int col0 = 32 * w;
+            const int sh = col0 - s;  // tree index of column col0
+            // prefix part
+            if (s >= col0 + 32) word = 0xFFFFFFFFu;
+            else if (s > col0) word = (1u << (s - col0)) - 1u;
+            // tree part: bits of the 128-bit anc starting at tree index sh
+            uint32_t tw = 0;
+            if (sh >= 0) {
+              const int wi = sh >> 5, bi = sh & 31;
+              const uint32_t lo = wi < 4 ? (wi == 0 ? anc[0] : wi == 1 ? anc[1] : wi == 2 ? anc[2] : anc[3]) : 0u;
+              const uint32_t hi = wi + 1 < 4 ? (wi == 0 ? anc[1] : wi == 1 ? anc[2] : anc[3]) : 0u;
+              tw = bi ? ((lo >> bi) | (hi << (32 - bi))) : lo;
+            } else if (sh > -32) {
+              tw = anc[0] << (-sh);
+            }
+            vis[w] = word | tw;
+          }
+        }
+        // row maximum of the visible scores (log2 domain)
+        float tmax = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int c = 0; c < 32; ++c) {
+            float v = __uint_as_float(sreg[q][c]) * p.scale_log2;
+            if (masked && !((vis[q] >> c) & 1u)) v = -INFINITY;
+            sreg[q][c] = __float_as_uint(v);
+            tmax = fmaxf(tmax, v);
+          }
+        // lazy rescale: keep the old reference unless the maximum grew by more than 2^8
+        float alpha = 1.f;
+        if (tmax > m_ref + 8.f) {
+          alpha = (m_ref == -INFINITY) ? 0.f : fast_exp2(m_ref - tmax);
+          m_ref = tmax;
+        }
+        const bool need = (alpha != 1.f) && (j > 0);
+        if (__any_sync(0xFFFFFFFFu, need)) {
+          // O of this unit holds tiles < j; PV(j-1) must have landed before it is rescaled
+          const uint32_t pb = (g - 1u) & 1u;
+          ok = mbar_wait(bar(BAR_PVDONE + pb), ((g - 1u) >> 1) & 1u, s_abort);
+          ok = __all_sync(0xFFFFFFFFu, ok);
+          if (!ok) break;
+          tc_fence_after();
+#pragma unroll
+          for (int q = 0; q < 4; ++q) {
+            uint32_t oreg[32];
+            tc_ld32(tmem + lane_base + 256u + ob * 128u + q * 32u, oreg);
+            tc_wait_ld();
+#pragma unroll
+            for (int c = 0; c < 32; ++c) oreg[c] = __float_as_uint(__uint_as_float(oreg[c]) * alpha);
+            tc_st32(tmem + lane_base + 256u + ob * 128u + q * 32u, oreg);
+          }
+        }
+        l *= alpha;
+        const float sub = (m_ref == -INFINITY) ? 0.f : m_ref;
+        float sum = 0.f;
+        uint32_t preg[2][32];
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+#pragma unroll
+          for (int c = 0; c < 32; c += 2) {
+            const float p0 = fast_exp2(__uint_as_float(sreg[q][c]) - sub);
+            const float p1 = fast_exp2(__uint_as_float(sreg[q][c + 1]) - sub);
+            sum += p0 + p1;
+            __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
+            preg[q >> 1][(q & 1) * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&pk);
+          }
+        l += sum;
+        tc_st32(tmem + lane_base + sb * 128u, preg[0]);
+        tc_st32(tmem + lane_base + sb * 128u + 32u, preg[1]);
+        tc_wait_st();
+        tc_fence_before();
+        mbar_arrive(bar(BAR_PFULL + sb));
+      }
+      if (!ok) break;
+      // ---- epilogue of the unit
+      float* po = p.part_o + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 128;
+      float* pml = p.part_ml + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 2;
+      if (nt <= 0) {  // empty split: contributes nothing
+        if (p.S > 1 && r < p.N) {
+          pml[0] = -INFINITY;
+          pml[1] = 0.f;
+        }
+        continue;
+      }
+      const uint32_t lb = (g - 1u) & 1u;
+      ok = mbar_wait(bar(BAR_PVDONE + lb), ((g - 1u) >> 1) & 1u, s_abort);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      tc_fence_after();
+      const float inv = 1.f / l;
+      __nv_bfloat16* orow = p.out + x.b * p.os_b + x.layer * p.os_l + x.h * p.os_h + static_cast<int64_t>(r) * p.os_t;
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t oreg[32];
+        tc_ld32(tmem + lane_base + 256u + ob * 128u + q * 32u, oreg);
+        tc_wait_ld();
+        if (q == 3) {  // the O buffer is in registers: hand it back to the MMA warp
+          tc_fence_before();
+          mbar_arrive(bar(BAR_OFREE + ob));
+        }
+        if (r < p.N) {
+          if (p.S == 1) {
+#pragma unroll
+            for (int c = 0; c < 32; c += 8) {
+              uint4 w;
+              __nv_bfloat162 t0 = __floats2bfloat162_rn(__uint_as_float(oreg[c + 0]) * inv, __uint_as_float(oreg[c + 1]) * inv);
+              __nv_bfloat162 t1 = __floats2bfloat162_rn(__uint_as_float(oreg[c + 2]) * inv, __uint_as_float(oreg[c + 3]) * inv);
+              __nv_bfloat162 t2 = __floats2bfloat162_rn(__uint_as_float(oreg[c + 4]) * inv, __uint_as_float(oreg[c + 5]) * inv);
+              __nv_bfloat162 t3 = __floats2bfloat162_rn(__uint_as_float(oreg[c + 6]) * inv, __uint_as_float(oreg[c + 7]) * inv);
+              w.x = *reinterpret_cast<uint32_t*>(&t0); w.y = *reinterpret_cast<uint32_t*>(&t1);
+              w.z = *reinterpret_cast<uint32_t*>(&t2); w.w = *reinterpret_cast<uint32_t*>(&t3);
+              *reinterpret_cast<uint4*>(orow + q * 32 + c) = w;
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 32; c += 4)
+              *reinterpret_cast<float4*>(po + q * 32 + c) =
+                  make_float4(__uint_as_float(oreg[c]), __uint_as_float(oreg[c + 1]), __uint_as_float(oreg[c + 2]),
+                              __uint_as_float(oreg[c + 3]));
+          }
+        }
+      }
+      if (p.S > 1 && r < p.N) {
+        pml[0] = m_ref;
+        pml[1] = l;
+      }
+      ++ui;
+    }
+  }
+
+  // ---- teardown: every thread arrives here, also after an aborted wait
+  __syncthreads();
+  if (*s_abort) {
+    if (tid == 0) atomicOr(p.flags, TR_FLAG_WAIT_TIMEOUT);
+    // give copies and MMAs that may still be in flight time to land before shared memory and TMEM are released
+    for (int i = 0; i < 200; ++i) __nanosleep(1000);
+    __syncthreads();
+  }
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (fn) return fn;
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess)
+    return nullptr;
+  fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  return fn;
+}
+
+// 5-D bf16 tensor map with 128-byte swizzle; out-of-bounds elements read as zero.  dims[0] is head_dim (contiguous);
+// strides (elements) belong to dims[1..4]; a stride of a size-1 dimension may be anything.
+bool encode_map(CUtensorMap* m, const void* ptr, const uint64_t (&dims)[5], const int64_t (&strides)[4],
+                const uint32_t (&box)[5]) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (!fn) return false;
+  cuuint64_t gd[5], gs[4];
+  cuuint32_t bx[5], es[5] = {1, 1, 1, 1, 1};
+  for (int i = 0; i < 5; ++i) { gd[i] = dims[i]; bx[i] = box[i]; }
+  for (int i = 0; i < 4; ++i) gs[i] = static_cast<cuuint64_t>(strides[i] > 0 ? strides[i] : HD) * 2;  // bytes
+  return fn(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(ptr), gd, gs, bx, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+tr_status tr_attention_tc_setup() {
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
+}
+
+void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
+
+tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s) {
+  if (a->head_dim != HD) return TR_ERR_UNSUPPORTED;
+  const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * a->n_q_heads;
+  if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
+  TcParams p;
+  p.out = static_cast<__nv_bfloat16*>(a->out);
+  p.ctx_len = a->d_ctx_len;
+  p.anc = ctx->d_anc;
+  p.part_o = ctx->d_attn_part_o;
+  p.part_ml = ctx->d_attn_part_ml;
+  p.flags = ctx->d_flags;
+  p.N = ctx->n_nodes; p.Hq = a->n_q_heads; p.Hkv = a->n_kv_heads; p.L = a->n_layers;
+  p.os_b = a->o_stride[0]; p.os_h = a->o_stride[1]; p.os_t = a->o_stride[2]; p.os_l = a->layer_stride_o;
+  const float scale = a->scale != 0.f ? a->scale : 1.0f / sqrtf(static_cast<float>(a->head_dim));
+  p.scale_log2 = scale * 1.4426950408889634f;
+  p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK);
+  p.n_units = static_cast<int>(base * p.S);
+
+  // Q is addressed as (dim, head, node, layer, sequence): in the usual [.., node, head, dim] layout the head
+  // stride is the smaller one, and the tile (64 dims x 1 head x 128 nodes) lands in shared memory as 128 rows.
+  CUtensorMap mq, mk, mv;
+  const uint64_t qd[5] = {HD, (uint64_t)a->n_q_heads, (uint64_t)ctx->n_nodes, (uint64_t)a->n_layers, (uint64_t)ctx->batch};
+  const int64_t qs[4] = {a->q_stride[1], a->q_stride[2], a->layer_stride_q, a->q_stride[0]};
+  const uint32_t qbox[5] = {64, 1, BK, 1, 1};
+  const uint64_t kd[5] = {HD, (uint64_t)a->kv_rows, (uint64_t)a->n_kv_heads, (uint64_t)a->n_layers, (uint64_t)ctx->batch};
+  const int64_t ks[4] = {a->kv_stride[2], a->kv_stride[1], a->layer_stride_kv, a->kv_stride[0]};
+  const uint32_t kbox[5] = {64, BK, 1, 1, 1};
+  if (!encode_map(&mq, a->q, qd, qs, qbox) || !encode_map(&mk, a->k_cache, kd, ks, kbox) ||
+      !encode_map(&mv, a->v_cache, kd, ks, kbox))
+    return TR_ERR_UNSUPPORTED;
+  const int grid = p.n_units < ctx->sm_count ? p.n_units : ctx->sm_count;
+  tr_attn_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+  TR_CUDA_TRY(cudaGetLastError());
+  if (p.S > 1) tr_launch_attention_combine(ctx, a, p.S, s);
+  TR_CUDA_TRY(cudaGetLastError());
+  return TR_OK;
+}

@@ -1,5 +1,6 @@
 // Host side of the C ABI: context, template validation and derived tables, matrix state, status.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -145,7 +146,10 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaDeviceSynchronize());
 #undef TR_INIT_TRY
   {
-    const tr_status st = tr_attention_mma_setup();
+    tr_status st = tr_attention_mma_setup();
+    if (st == TR_OK) st = tr_attention_tc_setup();
+    const char* force = getenv("TR_ATTN_FORCE_MMA");
+    c->force_mma = force && force[0] == '1';
     if (st != TR_OK) {
       free_all(c);
       return st;
@@ -240,6 +244,8 @@ static tr_status check_attn_args(const tr_ctx* ctx, const tr_attn_args* a) {
 extern "C" tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* a, void* stream) {
   tr_status st = check_attn_args(ctx, a);
   if (st != TR_OK) return st;
+  // head_dim 128 runs on the tcgen05 / TMA kernel; head_dim 64 on the warp-level MMA kernel
+  if (a->head_dim == 128 && !ctx->force_mma) return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
   return tr_launch_attention_mma(ctx, a, static_cast<cudaStream_t>(stream));
 }
 

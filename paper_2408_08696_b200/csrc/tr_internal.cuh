@@ -46,6 +46,7 @@ struct tr_ctx {
   float* d_attn_part_o = nullptr;   // [slots][128][128]
   float* d_attn_part_ml = nullptr;  // [slots][128][2]
   uint32_t* d_flags = nullptr;
+  bool force_mma = false;  // debugging aid: TR_ATTN_FORCE_MMA=1 at tr_init keeps head_dim 128 on the warp-MMA kernel
 };
 
 // launchers (host functions defined next to their kernels)
@@ -54,4 +55,7 @@ tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* 
 tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);
 tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_mma_setup();
+tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
+tr_status tr_attention_tc_setup();
+void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
 int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys);

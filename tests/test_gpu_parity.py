@@ -198,6 +198,7 @@ def _attention_case(harness, w, n_layers, splits=0):
                 mx, rel = attention_close(got[b, l, :, h], ref[:, h])
                 assert mx <= ATOL and rel <= RTOL, (b, l, h, mx, rel)
                 worst = (max(worst[0], mx), max(worst[1], rel))
+    assert tr.tr_device_flags(dw.ctx) == 0
     dw.close()
     return worst
 
@@ -250,6 +251,7 @@ def test_attention_llama2_7b_full_size_sampled(harness):
         mx, rel = attention_close(got, ref[:, 0])
         assert mx <= ATOL and rel <= RTOL, (l, h, mx, rel)
     assert torch.isfinite(dw.o.float()).all()
+    assert tr.tr_device_flags(dw.ctx) == 0
     dw.close()
 
 
