@@ -75,11 +75,15 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completes.
+// kBackoff: sleep a little between polls (the single-thread producer / MMA roles share their scheduler with a
+// softmax warp and should not take its issue slots).
+template <bool kBackoff = true>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    if (kBackoff) __nanosleep(40);
     if ((i & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
@@ -341,7 +345,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const uint32_t ob = ui & 1u;
       for (int j = 0; j < nt && ok; ++j, ++g) {
         const uint32_t sb = g & 1u;
-        ok = mbar_wait(bar(BAR_SFULL + sb), (g >> 1) & 1u, s_abort);
+        ok = mbar_wait<false>(bar(BAR_SFULL + sb), (g >> 1) & 1u, s_abort);
         ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
         if (!ok) break;
         tc_fence_after();
@@ -377,17 +381,23 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             vis[w] = word | tw;
           }
         }
-        // row maximum of the visible scores (log2 domain)
-        float tmax = -INFINITY;
+        if (masked) {  // only the one or two tiles that reach into the tree's keys
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+#pragma unroll
+            for (int c = 0; c < 32; ++c)
+              if (!((vis[q] >> c) & 1u)) sreg[q][c] = 0xFF800000u;  // -inf
+        }
+        // row maximum of the raw scores: eight independent chains (scale > 0, applied afterwards)
+        float mx[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mx[i] = -INFINITY;
 #pragma unroll
         for (int q = 0; q < 4; ++q)
 #pragma unroll
-          for (int c = 0; c < 32; ++c) {
-            float v = __uint_as_float(sreg[q][c]) * p.scale_log2;
-            if (masked && !((vis[q] >> c) & 1u)) v = -INFINITY;
-            sreg[q][c] = __float_as_uint(v);
-            tmax = fmaxf(tmax, v);
-          }
+          for (int c = 0; c < 32; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sreg[q][c]));
+        const float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
+                                 fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
         // lazy rescale: keep the old reference unless the maximum grew by more than 2^8
         float alpha = 1.f;
         if (tmax > m_ref + 8.f) {
@@ -398,7 +408,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (__any_sync(0xFFFFFFFFu, need)) {
           // O of this unit holds tiles < j; PV(j-1) must have landed before it is rescaled
           const uint32_t pb = (g - 1u) & 1u;
-          ok = mbar_wait(bar(BAR_PVDONE + pb), ((g - 1u) >> 1) & 1u, s_abort);
+          ok = mbar_wait<false>(bar(BAR_PVDONE + pb), ((g - 1u) >> 1) & 1u, s_abort);
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -413,19 +423,21 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           }
         }
         l *= alpha;
-        const float sub = (m_ref == -INFINITY) ? 0.f : m_ref;
-        float sum = 0.f;
+        const float nsub = (m_ref == -INFINITY) ? 0.f : -m_ref;
+        float sm4[4] = {0.f, 0.f, 0.f, 0.f};
         uint32_t preg[2][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
-            const float p0 = fast_exp2(__uint_as_float(sreg[q][c]) - sub);
-            const float p1 = fast_exp2(__uint_as_float(sreg[q][c + 1]) - sub);
-            sum += p0 + p1;
+            const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[q][c]), p.scale_log2, nsub));
+            const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[q][c + 1]), p.scale_log2, nsub));
+            sm4[(c >> 1) & 1] += p0;
+            sm4[2 + ((c >> 1) & 1)] += p1;
             __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
             preg[q >> 1][(q & 1) * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&pk);
           }
+        const float sum = (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
         l += sum;
         tc_st32(tmem + lane_base + sb * 128u, preg[0]);
         tc_st32(tmem + lane_base + sb * 128u + 32u, preg[1]);
@@ -445,7 +457,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         continue;
       }
       const uint32_t lb = (g - 1u) & 1u;
-      ok = mbar_wait(bar(BAR_PVDONE + lb), ((g - 1u) >> 1) & 1u, s_abort);
+      ok = mbar_wait<false>(bar(BAR_PVDONE + lb), ((g - 1u) >> 1) & 1u, s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();

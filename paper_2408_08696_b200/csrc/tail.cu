@@ -13,9 +13,28 @@
 
 constexpr int TAIL_THREADS = 128;
 
+// Template tables staged in shared memory once per kernel (one parallel fetch instead of dependent global loads).
+struct TailTables {
+  int32_t parent[TR_MAX_NODES];
+  int32_t rank[TR_MAX_NODES];
+  int32_t depth[TR_MAX_NODES];
+  int32_t level_off[TR_MAX_NODES + 2];
+};
+
+__device__ __forceinline__ void load_tables(TailTables& t, int n, int depth_max, const int32_t* __restrict__ parent,
+                                            const int32_t* __restrict__ rank, const int32_t* __restrict__ depth,
+                                            const int32_t* __restrict__ level_off, int tid) {
+  if (tid < n) {
+    t.parent[tid] = parent[tid];
+    t.rank[tid] = rank[tid];
+    t.depth[tid] = depth[tid];
+  }
+  for (int i = tid; i < depth_max + 2; i += TAIL_THREADS) t.level_off[i] = level_off[i];
+}
+
 __device__ __forceinline__ void bfs_expand(const int32_t* __restrict__ M, int V, int k, int n,
-                                           const int32_t* __restrict__ parent, const int32_t* __restrict__ rank,
-                                           const int32_t* __restrict__ level_off, int depth_max,
+                                           const int32_t* parent, const int32_t* rank,
+                                           const int32_t* level_off, int depth_max,
                                            int32_t* s_tree /* shared [n], s_tree[0] set */, int tid) {
   // one dependent round of gathers per level; every node of a level is looked up in parallel
   for (int d = 1; d <= depth_max; ++d) {
@@ -32,8 +51,10 @@ tr_build_tree_kernel(const int32_t* __restrict__ M_all, int V, int k, int n, con
                      const int32_t* __restrict__ rank, const int32_t* __restrict__ level_off, int depth_max,
                      const int32_t* __restrict__ root, int32_t* __restrict__ tree, uint32_t* __restrict__ flags) {
   __shared__ int32_t s_tree[TR_MAX_NODES];
+  __shared__ TailTables tb;
   const int b = blockIdx.x, tid = threadIdx.x;
   const int32_t* M = M_all + static_cast<size_t>(b) * V * k;
+  load_tables(tb, n, depth_max, parent, rank, rank, level_off, tid);
   if (tid == 0) {
     int32_t r = root[b];
     if (r < 0 || r >= V) {
@@ -42,7 +63,7 @@ tr_build_tree_kernel(const int32_t* __restrict__ M_all, int V, int k, int n, con
     }
     s_tree[0] = r;
   }
-  bfs_expand(M, V, k, n, parent, rank, level_off, depth_max, s_tree, tid);
+  bfs_expand(M, V, k, n, tb.parent, tb.rank, tb.level_off, depth_max, s_tree, tid);
   if (tid < n) tree[static_cast<size_t>(b) * n + tid] = s_tree[tid];
 }
 
@@ -57,7 +78,9 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   __shared__ int32_t s_argmax[TR_MAX_NODES];
   __shared__ int32_t s_tree[TR_MAX_NODES];
   __shared__ uint32_t s_best[TAIL_THREADS / 32];
+  __shared__ TailTables tb;
   const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  load_tables(tb, n, depth_max, parent, rank, depth, level_off, tid);
   int32_t* M = M_all + static_cast<size_t>(b) * V * k;
   const int32_t* topk = topk_idx + static_cast<size_t>(b) * n * k;
   const int W = depth_max + 1;
@@ -78,12 +101,12 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   if (tid < n) {
     bool ok = true;
     for (int x = tid; x > 0;) {
-      const int p = parent[x];
+      const int p = tb.parent[x];
       ok = ok && (s_S[x] == s_argmax[p]);
       x = p;
     }
     // deeper first, then lower index; +1 keeps every valid key above the 0 of idle threads
-    if (ok) keyv = (static_cast<uint32_t>(depth[tid]) << 8 | static_cast<uint32_t>(255 - tid)) + 1u;
+    if (ok) keyv = (static_cast<uint32_t>(tb.depth[tid]) << 8 | static_cast<uint32_t>(255 - tid)) + 1u;
   }
   const uint32_t wbest = __reduce_max_sync(0xFFFFFFFFu, keyv);
   if (lane == 0) s_best[warp] = wbest;
@@ -102,7 +125,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     for (int d = acc_len; d >= 0; --d) {  // fill the path backwards
       acc_nodes[b * W + d] = x;
       if (d > 0) out_tokens[b * W + d - 1] = s_S[x];
-      x = parent[x];
+      x = tb.parent[x];
     }
     out_tokens[b * W + acc_len] = bonus;
     for (int d = acc_len + 1; d < W; ++d) {
@@ -123,7 +146,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     }
   }
   // ---- retrieve the next tree from the updated matrix (bfs_expand starts with a __syncthreads())
-  bfs_expand(M, V, k, n, parent, rank, level_off, depth_max, s_tree, tid);
+  bfs_expand(M, V, k, n, tb.parent, tb.rank, tb.level_off, depth_max, s_tree, tid);
   if (tid < n) tree_out[static_cast<size_t>(b) * n + tid] = s_tree[tid];
 }
 

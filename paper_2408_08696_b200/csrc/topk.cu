@@ -12,6 +12,7 @@
 #include "tr_internal.cuh"
 
 typedef unsigned long long u64;
+constexpr int TOPK_MERGE_CAP = 1024;
 
 __device__ __forceinline__ u64 topk_key(float v, uint32_t idx) {
   uint32_t b = __float_as_uint(v);
@@ -51,6 +52,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   __shared__ u64 s_wtop[NW * TR_MAX_K];
   __shared__ u64 s_cand[TR_MAX_K * E];
   __shared__ u64 s_out[TR_MAX_K];
+  __shared__ u64 s_merge[TOPK_MERGE_CAP];
   __shared__ int s_cnt;
   __shared__ int s_last;
 
@@ -138,14 +140,19 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   __syncthreads();
   if (!s_last) return;
   __threadfence();
+  const u64* row_part = part + static_cast<size_t>(row) * segs * k;
+  const int n = segs * k;
+  const bool staged = n <= TOPK_MERGE_CAP;  // one parallel fetch of every partial list, then rounds in shared memory
+  if (staged) {
+    for (int i = tid; i < n; i += TOPK_THREADS) s_merge[i] = __ldcg(row_part + i);
+    __syncthreads();
+  }
   if (warp == 0) {
-    const u64* row_part = part + static_cast<size_t>(row) * segs * k;
-    const int n = segs * k;
     u64 last = ~0ull;
     for (int r = 0; r < k; ++r) {
       u64 best = 0;
       for (int i = lane; i < n; i += 32) {
-        const u64 x = __ldcg(row_part + i);
+        const u64 x = staged ? s_merge[i] : __ldcg(row_part + i);
         if (x < last && x > best) best = x;
       }
       last = warp_max_u64(best);

@@ -226,6 +226,7 @@ static tr_status check_attn_args(const tr_ctx* ctx, const tr_attn_args* a) {
   if (!ctx || !a || !a->q || !a->k_cache || !a->v_cache || !a->out || !a->d_ctx_len) return TR_ERR_INVALID_ARG;
   if (a->n_q_heads < 1 || a->n_kv_heads < 1 || a->n_q_heads % a->n_kv_heads != 0) return TR_ERR_INVALID_ARG;
   if (a->head_dim != 64 && a->head_dim != 128) return TR_ERR_UNSUPPORTED;
+  if (!(a->scale >= 0.f) || a->scale > 1e30f) return TR_ERR_INVALID_ARG;  // 0 selects 1/sqrt(head_dim)
   if (a->n_layers < 1 || a->max_ctx < 0 || a->kv_rows < a->max_ctx + ctx->n_nodes || a->splits < 0)
     return TR_ERR_INVALID_ARG;
   const uintptr_t ptrs[4] = {(uintptr_t)a->q, (uintptr_t)a->k_cache, (uintptr_t)a->v_cache, (uintptr_t)a->out};
