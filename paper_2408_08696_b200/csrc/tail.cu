@@ -86,13 +86,16 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   const int W = depth_max + 1;
 
   int32_t tok = 0;
+  int32_t row[TR_MAX_K];
   bool tok_ok = false;
   if (tid < n) {
     tok = tree_in[static_cast<size_t>(b) * n + tid];
     tok_ok = (tok >= 0 && tok < V);
     if (!tok_ok) atomicOr(flags, TR_FLAG_BAD_TOKEN);
     s_S[tid] = tok;
-    s_argmax[tid] = topk[tid * k];
+#pragma unroll
+    for (int c = 0; c < TR_MAX_K; ++c) row[c] = c < k ? topk[tid * k + c] : 0;  // fetched once, with the tokens
+    s_argmax[tid] = row[0];
   }
   __syncthreads();
 
@@ -141,8 +144,9 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     for (int j = tid + 1; j < n; ++j) last = last && (s_S[j] != tok);
     if (last) {
       int32_t* dst = M + static_cast<size_t>(tok) * k;
-      const int32_t* src = topk + tid * k;
-      for (int c = 0; c < k; ++c) dst[c] = src[c];
+#pragma unroll
+      for (int c = 0; c < TR_MAX_K; ++c)
+        if (c < k) dst[c] = row[c];
     }
   }
   // ---- retrieve the next tree from the updated matrix (bfs_expand starts with a __syncthreads())

@@ -5,14 +5,15 @@
 // keys" - any split / merge order gives the same answer, bit for bit.
 //
 // A logits row is cut into segments of TOPK_SEG_ELEMS; one CTA per (segment, row) keeps its 16 values per
-// thread in registers (128-bit loads), finds a threshold that is guaranteed not to exceed the segment's
-// k-th largest key (the k-th largest of the per-thread maxima), collects the few keys at or above it and
-// selects the segment's top-k exactly.  The last CTA of a row to finish (atomic ticket, no waiting) merges the
-// per-segment lists into the row's final top-k.
+// thread in registers (128-bit loads), finds a threshold that cannot exceed the segment's k-th largest key
+// (the k-th largest of the 16 half-warp maxima), collects the few keys at or above it - only threads whose own
+// maximum reaches the threshold look at all - and selects the segment's top-k exactly.  The last CTA of a row
+// to finish (atomic ticket, no waiting) merges the per-segment lists into the row's final top-k.
 #include "tr_internal.cuh"
 
 typedef unsigned long long u64;
 constexpr int TOPK_MERGE_CAP = 1024;
+constexpr int TOPK_CAND_CAP = 512;
 
 __device__ __forceinline__ u64 topk_key(float v, uint32_t idx) {
   uint32_t b = __float_as_uint(v);
@@ -28,18 +29,17 @@ __device__ __forceinline__ u64 warp_max_u64(u64 x) {
   return (static_cast<u64>(mh) << 32) | ml;
 }
 
-// The k largest keys of arr[0..n) in descending order, one warp; out[r] = 0 when fewer than r+1 keys exist.
-// Each round takes the largest key strictly below the previous winner (keys are distinct).
-__device__ __forceinline__ void warp_select_topk(const u64* arr, int n, int k, u64* out, int lane) {
+// The k largest keys of s_in[0..n) (n may be 0) in descending order into out[0..k), one warp; missing entries 0.
+__device__ __forceinline__ void warp_rounds(const u64* s_in, int n, int k, u64* out, int lane) {
   u64 last = ~0ull;
   for (int r = 0; r < k; ++r) {
     u64 best = 0;
     for (int i = lane; i < n; i += 32) {
-      const u64 x = arr[i];
+      const u64 x = s_in[i];
       if (x < last && x > best) best = x;
     }
     last = warp_max_u64(best);
-    if (lane == 0) out[r] = last;  // once 0 (nothing left) it stays 0
+    if (lane == 0) out[r] = last;
   }
 }
 
@@ -48,11 +48,12 @@ __global__ void __launch_bounds__(TOPK_THREADS)
 tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __restrict__ part,
                unsigned int* __restrict__ ticket, int32_t* __restrict__ topk_idx) {
   constexpr int E = TOPK_ELEMS_PER_THREAD;
-  constexpr int NW = TOPK_THREADS / 32;
-  __shared__ u64 s_wtop[NW * TR_MAX_K];
-  __shared__ u64 s_cand[TR_MAX_K * E];
+  constexpr int G = TOPK_THREADS / 16;  // half-warp groups: 16 >= TR_MAX_K
+  __shared__ u64 s_gmax[G];
+  __shared__ u64 s_cand[TOPK_CAND_CAP];
   __shared__ u64 s_out[TR_MAX_K];
   __shared__ u64 s_merge[TOPK_MERGE_CAP];
+  __shared__ u64 s_tau;
   __shared__ int s_cnt;
   __shared__ int s_last;
 
@@ -62,75 +63,104 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   const float* rowp = logits + static_cast<size_t>(row) * V;
   const int seg_base = seg * TOPK_SEG_ELEMS;
 
-  u64 key[E];
+  // ---- (1) 16 values per thread in registers; running maximum with its index (first = lowest index wins ties)
+  float v[E];
+  int idx0[E / 4];  // index of each 4-group's first element (vector path) -- scalar path uses j * THREADS + tid
   if (kVec) {
-    float4 v[E / 4];
 #pragma unroll
     for (int j = 0; j < E / 4; ++j) {
       const int i0 = seg_base + j * (TOPK_THREADS * 4) + tid * 4;
-      v[j] = (i0 < V) ? __ldcs(reinterpret_cast<const float4*>(rowp + i0)) : make_float4(0, 0, 0, 0);
-    }
-#pragma unroll
-    for (int j = 0; j < E / 4; ++j) {
-      const int i0 = seg_base + j * (TOPK_THREADS * 4) + tid * 4;
-      const bool ok = i0 < V;  // V % 4 == 0 on this path
-      key[4 * j + 0] = ok ? topk_key(v[j].x, i0 + 0) : 0ull;
-      key[4 * j + 1] = ok ? topk_key(v[j].y, i0 + 1) : 0ull;
-      key[4 * j + 2] = ok ? topk_key(v[j].z, i0 + 2) : 0ull;
-      key[4 * j + 3] = ok ? topk_key(v[j].w, i0 + 3) : 0ull;
+      idx0[j] = i0;
+      float4 t = (i0 < V) ? __ldcs(reinterpret_cast<const float4*>(rowp + i0))
+                          : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
     }
   } else {
-    float v[E];
 #pragma unroll
     for (int j = 0; j < E; ++j) {
       const int i = seg_base + j * TOPK_THREADS + tid;
-      v[j] = (i < V) ? __ldcs(rowp + i) : 0.f;
-    }
-#pragma unroll
-    for (int j = 0; j < E; ++j) {
-      const int i = seg_base + j * TOPK_THREADS + tid;
-      key[j] = (i < V) ? topk_key(v[j], i) : 0ull;
+      v[j] = (i < V) ? __ldcs(rowp + i) : -INFINITY;
     }
   }
+  auto index_of = [&](int j) -> int {
+    return kVec ? idx0[j >> 2] + (j & 3) : seg_base + j * TOPK_THREADS + tid;
+  };
   if (tid == 0) s_cnt = 0;
+  float bv = v[0];
+  int bj = 0;
+#pragma unroll
+  for (int j = 1; j < E; ++j)
+    if (v[j] > bv) { bv = v[j]; bj = j; }  // -0 == +0 here as well; indices ascend with j
+  int bi = 0;
+#pragma unroll
+  for (int j = 0; j < E; ++j) bi = (bj == j) ? index_of(j) : bi;
+  const u64 tmax = (bi < V) ? topk_key(bv, bi) : 0ull;  // padding threads past the row's end hold no key
 
-  // (1) per-thread maximum, (2) each warp's k largest thread maxima
-  u64 tmax = 0;
-#pragma unroll
-  for (int j = 0; j < E; ++j) tmax = key[j] > tmax ? key[j] : tmax;
+  // ---- (2) maxima of the 16 half-warp groups; threshold = k-th largest of them.  At least k keys of the segment
+  //          are >= it, so the segment's top-k lies among the keys >= it.
   {
-    u64 cur = tmax;
+    const unsigned mask = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
+    const uint32_t hi = static_cast<uint32_t>(tmax >> 32), lo = static_cast<uint32_t>(tmax);
+    const uint32_t mh = __reduce_max_sync(mask, hi);
+    const uint32_t ml = __reduce_max_sync(mask, hi == mh ? lo : 0u);
+    if ((lane & 15) == 0) s_gmax[tid >> 4] = (static_cast<u64>(mh) << 32) | ml;
+  }
+  __syncthreads();
+  if (warp == 0) {
+    u64 tau = ~0ull;
+    const u64 mine = lane < G ? s_gmax[lane] : 0ull;
     for (int r = 0; r < k; ++r) {
-      const u64 w = warp_max_u64(cur);
-      if (lane == r) s_wtop[warp * k + r] = w;
-      if (cur == w) cur = 0;  // the (unique) winner retires; if w == 0 nothing changes
+      tau = warp_max_u64(mine < tau ? mine : 0ull);
+      if (tau == 0) break;  // fewer than k non-empty groups: every key is a candidate
     }
+    if (lane == 0) s_tau = tau;
   }
   __syncthreads();
-  // (3) threshold = k-th largest thread maximum of the CTA: at least k keys of the segment are >= it, and
-  //     only the <= k threads holding those maxima can hold keys >= it, so at most k*E candidates follow.
-  u64 tau = ~0ull;
-  for (int r = 0; r < k; ++r) {
-    u64 best = 0;
-    for (int i = lane; i < NW * k; i += 32) {
-      const u64 x = s_wtop[i];
-      if (x < tau && x > best) best = x;
-    }
-    tau = warp_max_u64(best);
-    if (tau == 0) break;  // fewer than k non-empty threads: every valid key is a candidate
-  }
+  // ---- (3) candidates: only threads whose own maximum reaches the threshold look at their values
+  const u64 tau = s_tau;
+  if (tmax != 0 && tmax >= tau) {
 #pragma unroll
-  for (int j = 0; j < E; ++j) {
-    if (key[j] != 0 && key[j] >= tau) {
-      const int p = atomicAdd(&s_cnt, 1);
-      s_cand[p] = key[j];
+    for (int j = 0; j < E; ++j) {
+      const int i = index_of(j);
+      if (i < V) {
+        const u64 key = topk_key(v[j], i);
+        if (key >= tau) {
+          const int p = atomicAdd(&s_cnt, 1);
+          if (p < TOPK_CAND_CAP) s_cand[p] = key;
+        }
+      }
     }
   }
   __syncthreads();
-  // (4) exact top-k of the candidates -> this segment's partial list
+  // ---- (4) exact top-k of the candidates -> this segment's partial list
   u64* my_part = part + (static_cast<size_t>(row) * segs + seg) * k;
-  if (warp == 0) warp_select_topk(s_cand, s_cnt, k, my_part, lane);
-  // (5) ticket: the last CTA of the row merges all partial lists
+  const int cnt = s_cnt;
+  if (cnt <= TOPK_CAND_CAP) {
+    if (warp == 0) warp_rounds(s_cand, cnt, k, my_part, lane);
+  } else {
+    // More candidates than the buffer holds (only with massive ties or adversarial layouts): select straight
+    // from the registers, round by round, the whole CTA taking part.
+    u64 last = ~0ull;
+    for (int r = 0; r < k; ++r) {
+      u64 best = 0;
+#pragma unroll
+      for (int j = 0; j < E; ++j) {
+        const int i = index_of(j);
+        const u64 key = (i < V) ? topk_key(v[j], i) : 0ull;
+        if (key < last && key > best) best = key;
+      }
+      best = warp_max_u64(best);
+      __syncthreads();  // previous round's readers are done with s_gmax
+      if (lane == 0) s_gmax[warp] = best;
+      __syncthreads();
+      u64 m = 0;
+#pragma unroll
+      for (int w = 0; w < TOPK_THREADS / 32; ++w) m = s_gmax[w] > m ? s_gmax[w] : m;
+      last = m;
+      if (tid == 0) my_part[r] = m;
+    }
+  }
+  // ---- (5) ticket: the last CTA of the row merges all partial lists
   __syncthreads();
   if (tid == 0) {
     __threadfence();

@@ -75,6 +75,15 @@ def test_topk_ties_and_special_values(tr, V):
     assert (_topk_case(tr, x, 8) == orc.argtopk(x, 8)).all()
 
 
+def test_topk_all_equal_rows_k16_take_the_overflow_path(tr):
+    # 16 candidates per token and constant rows: more keys reach the threshold than the candidate buffer holds
+    V = 9000
+    x = np.zeros((15, V), dtype=np.float32)
+    x[1] = -np.inf
+    x[2, 100:] = 1.0
+    assert (_topk_case(tr, x, 16) == orc.argtopk(x, 16)).all()
+
+
 def test_topk_adversarial_all_top_in_one_thread(tr):
     # every one of a thread's 16 register slots beats the rest of the segment: the candidate buffer's bound
     V = 8192
