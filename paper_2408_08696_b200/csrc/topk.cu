@@ -29,22 +29,8 @@ __device__ __forceinline__ u64 warp_max_u64(u64 x) {
   return (static_cast<u64>(mh) << 32) | ml;
 }
 
-// The k largest keys of s_in[0..n) (n may be 0) in descending order into out[0..k), one warp; missing entries 0.
-__device__ __forceinline__ void warp_rounds(const u64* s_in, int n, int k, u64* out, int lane) {
-  u64 last = ~0ull;
-  for (int r = 0; r < k; ++r) {
-    u64 best = 0;
-    for (int i = lane; i < n; i += 32) {
-      const u64 x = s_in[i];
-      if (x < last && x > best) best = x;
-    }
-    last = warp_max_u64(best);
-    if (lane == 0) out[r] = last;
-  }
-}
-
 template <bool kVec>
-__global__ void __launch_bounds__(TOPK_THREADS)
+__global__ void __launch_bounds__(TOPK_THREADS, 5)
 tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __restrict__ part,
                unsigned int* __restrict__ ticket, int32_t* __restrict__ topk_idx) {
   constexpr int E = TOPK_ELEMS_PER_THREAD;
@@ -53,7 +39,6 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   __shared__ u64 s_cand[TOPK_CAND_CAP];
   __shared__ u64 s_out[TR_MAX_K];
   __shared__ u64 s_merge[TOPK_MERGE_CAP];
-  __shared__ u64 s_tau;
   __shared__ int s_cnt;
   __shared__ int s_last;
 
@@ -106,18 +91,21 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
     if ((lane & 15) == 0) s_gmax[tid >> 4] = (static_cast<u64>(mh) << 32) | ml;
   }
   __syncthreads();
-  if (warp == 0) {
-    u64 tau = ~0ull;
+  // rank by counting, done by every warp for itself: the group maximum that has exactly k-1 larger ones is the
+  // threshold; with fewer than k non-empty groups the threshold is 0 and every key is a candidate
+  u64 tau;
+  {
     const u64 mine = lane < G ? s_gmax[lane] : 0ull;
-    for (int r = 0; r < k; ++r) {
-      tau = warp_max_u64(mine < tau ? mine : 0ull);
-      if (tau == 0) break;  // fewer than k non-empty groups: every key is a candidate
-    }
-    if (lane == 0) s_tau = tau;
+    int larger = 0;
+#pragma unroll
+    for (int i = 0; i < G; ++i) larger += (s_gmax[i] > mine) ? 1 : 0;
+    const unsigned hit = __ballot_sync(0xFFFFFFFFu, lane < G && mine != 0ull && larger == k - 1);
+    const int src = hit ? (__ffs(hit) - 1) : 0;
+    const uint32_t th = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(mine >> 32), src);
+    const uint32_t tl = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(mine), src);
+    tau = hit ? ((static_cast<u64>(th) << 32) | tl) : 0ull;
   }
-  __syncthreads();
   // ---- (3) candidates: only threads whose own maximum reaches the threshold look at their values
-  const u64 tau = s_tau;
   if (tmax != 0 && tmax >= tau) {
 #pragma unroll
     for (int j = 0; j < E; ++j) {
@@ -136,7 +124,20 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   u64* my_part = part + (static_cast<size_t>(row) * segs + seg) * k;
   const int cnt = s_cnt;
   if (cnt <= TOPK_CAND_CAP) {
-    if (warp == 0) warp_rounds(s_cand, cnt, k, my_part, lane);
+    // rank by counting: candidate with r larger ones is the segment's r-th entry; unused entries are 0
+    for (int t = tid; t < cnt; t += TOPK_THREADS) {
+      const u64 mine = s_cand[t];
+      int larger = 0;
+      for (int i = 0; i < cnt; ++i) larger += (s_cand[i] > mine) ? 1 : 0;
+      if (larger < k) {
+        my_part[larger] = mine;
+        __threadfence();  // published device-wide before this CTA takes its ticket
+      }
+    }
+    if (tid >= cnt && tid < k) {
+      my_part[tid] = 0ull;
+      __threadfence();
+    }
   } else {
     // More candidates than the buffer holds (only with massive ties or adversarial layouts): select straight
     // from the registers, round by round, the whole CTA taking part.
@@ -177,12 +178,23 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
     for (int i = tid; i < n; i += TOPK_THREADS) s_merge[i] = __ldcg(row_part + i);
     __syncthreads();
   }
-  if (warp == 0) {
+  if (staged) {
+    // every partial key counts the keys above it; the k keys with fewer than k above them are the answer
+    for (int t = tid; t < n; t += TOPK_THREADS) {
+      const u64 mine = s_merge[t];
+      if (mine == 0ull) continue;
+      int larger = 0;
+      for (int i = 0; i < n; ++i) larger += (s_merge[i] > mine) ? 1 : 0;
+      if (larger < k)
+        topk_idx[static_cast<size_t>(row) * k + larger] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(mine));
+    }
+    if (tid == 0) ticket[row] = 0u;  // ready for the next launch
+  } else if (warp == 0) {
     u64 last = ~0ull;
     for (int r = 0; r < k; ++r) {
       u64 best = 0;
       for (int i = lane; i < n; i += 32) {
-        const u64 x = staged ? s_merge[i] : __ldcg(row_part + i);
+        const u64 x = __ldcg(row_part + i);
         if (x < last && x > best) best = x;
       }
       last = warp_max_u64(best);
@@ -191,7 +203,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
     __syncwarp();
     if (lane < k) topk_idx[static_cast<size_t>(row) * k + lane] =
         static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(s_out[lane]));
-    if (lane == 0) ticket[row] = 0u;  // ready for the next launch
+    if (lane == 0) ticket[row] = 0u;
   }
 }
 
