@@ -178,6 +178,32 @@ typedef struct {
 tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_step_out* d_out, const tr_host_io* io,
                        void* stream);
 
+/*
+ * Top-k without any allocation (the paper has no counterpart; this entry point exists for deployment reasons).
+ *
+ * Who needs it: code that must not, or cannot, allocate device memory - for example a plug-in inside a serving
+ * process whose memory pool already owns all of HBM, so that cudaMalloc fails, or a latency-critical loop that
+ * cannot afford the device-wide synchronisation cudaMalloc and cudaFree imply.  tr_init allocates, so these
+ * callers cannot hold a context; this function needs none.
+ *
+ * What it computes: exactly the top-k part of tr_verify_update - for each of `rows` logits rows the indices of the
+ * k largest values, largest first, equal values by lower index (Sec. 2.1) - with the same kernel.  Its scratch
+ * (per-segment candidate lists and per-row tickets) lives in a fixed 528 KB device array inside the library,
+ * held by every GPU that loads the library until the process exits.
+ * DEVICE in : d_logits [rows, vocab] fp32 row-major.   DEVICE out: d_topk_idx [rows, k] int32.
+ * Limits    : rows <= 4096 and rows * ceil(vocab / 4096) * k <= 65536 (tr_topk_noalloc_limits reports both);
+ *             anything larger returns TR_ERR_UNSUPPORTED and launches nothing.  1 <= k <= TR_MAX_K <= vocab.
+ * The call allocates nothing and frees nothing; it enqueues one small memset and one kernel on `stream`.
+ * First call on a device: it asks the runtime for the device address of the array (once per device, with that
+ * device current).  Make this first call outside any stream capture.
+ * Sharing  : all calls on a device use the same array.  Calls issued to one stream are safe back to back (the
+ * tickets are cleared at the start of each call); calls that may overlap on the GPU (different streams, or
+ * different host threads feeding different streams) race on it and must be serialised by the caller.
+ */
+tr_status tr_topk_noalloc(const float* d_logits, int32_t rows, int32_t vocab, int32_t k, int32_t* d_topk_idx,
+                          void* stream);
+tr_status tr_topk_noalloc_limits(int32_t* max_rows, int32_t* max_partial_keys); /* HOST out */
+
 #ifdef __cplusplus
 }
 #endif

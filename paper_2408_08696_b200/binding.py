@@ -77,6 +77,8 @@ lib.tr_max_new_tokens.argtypes = [C.c_void_p]
 lib.tr_device_flags.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
 lib.tr_step_host.argtypes = [C.c_void_p, C.POINTER(tr_attn_args), C.POINTER(tr_step_out), C.POINTER(tr_host_io),
                              C.c_void_p]
+lib.tr_topk_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
+lib.tr_topk_noalloc_limits.argtypes = [_P32, _P32]
 lib_synth.trs_patch_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                        C.c_int32, C.c_int32, C.c_void_p]
 
@@ -238,6 +240,28 @@ def tr_device_flags(ctx):
 def tr_step_host(ctx, args, out_struct, io, stream=None):
     _check(lib.tr_step_host(ctx.handle, C.byref(args), C.byref(out_struct), C.byref(io), _stream(stream)),
            "tr_step_host")
+
+
+def tr_topk_noalloc_limits():
+    a, b = C.c_int32(0), C.c_int32(0)
+    _check(lib.tr_topk_noalloc_limits(C.byref(a), C.byref(b)), "tr_topk_noalloc_limits")
+    return a.value, b.value
+
+
+def tr_topk_noalloc(d_logits, k, d_topk_idx, stream=None):
+    """Top-k of every row of d_logits [rows, vocab] (fp32, contiguous) into d_topk_idx [rows, k] (int32) without a
+    context and without allocating: for callers that cannot call cudaMalloc.  The first call on a device should
+    happen outside stream capture; calls that overlap on the GPU share one scratch array and must be serialised."""
+    if d_logits.dim() != 2 or not d_logits.is_contiguous() or tuple(d_topk_idx.shape) != (d_logits.shape[0], k) \
+            or not d_topk_idx.is_contiguous():
+        raise ValueError("d_logits must be contiguous [rows, vocab] and d_topk_idx contiguous [rows, k]")
+    rows, vocab = d_logits.shape
+    st = lib.tr_topk_noalloc(_dev(d_logits, torch.float32, "d_logits"), rows, vocab, k,
+                             _dev(d_topk_idx, torch.int32, "d_topk_idx"), _stream(stream))
+    if st == TR_ERR_UNSUPPORTED:
+        mr, mp = tr_topk_noalloc_limits()
+        raise TrError(st, "tr_topk_noalloc: beyond the fixed scratch (rows <= %d, rows*segments*k <= %d)" % (mr, mp))
+    _check(st, "tr_topk_noalloc")
 
 
 def trs_patch_logits(d_logits, d_noise, d_tree, d_prev_col, d_succ, boost, stream=None):

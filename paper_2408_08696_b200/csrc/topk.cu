@@ -220,3 +220,70 @@ tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx
   TR_CUDA_TRY(cudaGetLastError());
   return TR_OK;
 }
+
+// ---------------------------------------------------------------------------------------------------
+// tr_topk_noalloc: the same kernel with its scratch in a fixed device array instead of context memory.
+//
+// Some callers of this library cannot allocate device memory at all: a plug-in running inside a serving
+// process that has handed every byte of HBM to its own pool (cudaMalloc simply fails there), or code on a
+// latency-critical path where the implicit device-wide synchronisation of cudaMalloc / cudaFree is not
+// acceptable.  tr_init allocates, so such callers cannot even create a context.  For them the per-segment
+// candidate lists and the per-row tickets of the top-k kernel live in the file-scope array below, which every
+// device that loads this library carries until the process exits.
+constexpr int NOALLOC_MAX_ROWS = 4096;            // logits rows per call
+constexpr int NOALLOC_MAX_PART = 65536;           // rows * segments * k partial keys per call
+constexpr size_t NOALLOC_TICKET_BYTES = sizeof(unsigned int) * NOALLOC_MAX_ROWS;
+constexpr size_t NOALLOC_BYTES = NOALLOC_TICKET_BYTES + sizeof(u64) * NOALLOC_MAX_PART;  // 528 KB
+
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
+
+#include <mutex>
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mutex;
+unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};  // device address of the array, per device
+}  // namespace
+
+extern "C" tr_status tr_topk_noalloc_limits(int32_t* max_rows, int32_t* max_partial_keys) {
+  if (!max_rows || !max_partial_keys) return TR_ERR_INVALID_ARG;
+  *max_rows = NOALLOC_MAX_ROWS;
+  *max_partial_keys = NOALLOC_MAX_PART;
+  return TR_OK;
+}
+
+extern "C" tr_status tr_topk_noalloc(const float* d_logits, int32_t rows, int32_t vocab, int32_t k,
+                                     int32_t* d_topk_idx, void* stream) {
+  if (!d_logits || !d_topk_idx || rows < 1 || k < 1 || k > TR_MAX_K || vocab < k) return TR_ERR_INVALID_ARG;
+  const int segs = (vocab + TOPK_SEG_ELEMS - 1) / TOPK_SEG_ELEMS;
+  if (rows > NOALLOC_MAX_ROWS || static_cast<int64_t>(rows) * segs * k > NOALLOC_MAX_PART || rows > 65535)
+    return TR_ERR_UNSUPPORTED;  // beyond the fixed scratch: see tr_topk_noalloc_limits
+  int dev = -1;
+  TR_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return TR_ERR_UNSUPPORTED;
+  unsigned char* base = nullptr;
+  {
+    // First call on this device: look up where this device keeps its copy of the array.  In host code the
+    // array's name is only a handle; the kernel must be given the address the runtime reports for it.
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+      void* p = nullptr;
+      TR_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
+      g_noalloc_ptr[dev] = static_cast<unsigned char*>(p);
+    }
+    base = g_noalloc_ptr[dev];
+  }
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned int* ticket = reinterpret_cast<unsigned int*>(base);
+  u64* part = reinterpret_cast<u64*>(base + NOALLOC_TICKET_BYTES);
+  // The array keeps whatever the previous call left behind.  The tickets must start at zero; the partial lists
+  // are fully rewritten by every call before they are read.
+  TR_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int) * rows, s));
+  const dim3 grid(segs, rows);
+  const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
+  if (vec)
+    tr_topk_kernel<true><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx);
+  else
+    tr_topk_kernel<false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx);
+  TR_CUDA_TRY(cudaGetLastError());
+  return TR_OK;
+}
