@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_TR_PATH = os.path.join(_PKG, "libtr.so")
+LIB_TR_PATH = os.environ.get("TR_LIB_PATH") or os.path.join(_PKG, "libtr.so")  # override: debugging aid
 LIB_SYNTH_PATH = os.path.join(_PKG, "libtr_synth.so")
 
 if not os.path.exists(LIB_TR_PATH) or not os.path.exists(LIB_SYNTH_PATH):

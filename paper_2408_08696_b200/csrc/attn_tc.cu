@@ -101,6 +101,21 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
       : "memory");
 }
+// Same load with an L2 eviction-priority hint: K/V tiles are read exactly once, so they are marked evict-first
+// and do not push the small, re-used state of the step (matrix rows, tables, logits) out of L2.
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+__device__ __forceinline__ void tma_load_5d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
+                                                 int c2, int c3, int c4, uint64_t pol) {
+  asm volatile(
+      "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, "
+      "{%3, %4, %5, %6, %7}], [%2], %8;"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "l"(pol)
+      : "memory");
+}
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
@@ -233,6 +248,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (lane == 0) {
       uint32_t ui = 0, c = 0;  // non-empty units done by this CTA; ring entries issued
       bool ok = true;
+      const uint64_t pol = l2_policy_evict_first();
       for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
         const Unit x = decode_unit(p, u);
         if (x.t0 >= x.t1) continue;
@@ -251,8 +267,8 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const CUtensorMap* m = kv == 0 ? &map_k : &map_v;
             const uint32_t dst = base + SM_RING + slot * TILE_BYTES;
             mbar_expect_tx(bar(BAR_FULL + slot), TILE_BYTES);
-            tma_load_5d(dst, m, bar(BAR_FULL + slot), 0, t * BK, x.kvh, x.layer, x.b);
-            tma_load_5d(dst + HALF_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b);
+            tma_load_5d_hint(dst, m, bar(BAR_FULL + slot), 0, t * BK, x.kvh, x.layer, x.b, pol);
+            tma_load_5d_hint(dst + HALF_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b, pol);
             ++c;
           }
         }
