@@ -1,11 +1,12 @@
 // Tree attention (paper Sec. 2.2) for head_dim 128 on the 5th-generation tensor cores: a persistent,
 // warp-specialised flash-decoding kernel.
 //
-//   warp 0      TMA producer: Q tile (double-buffered) and a ring of 32 KB K / V tiles (128 keys x 128 dims, bf16,
+//   warps 0..3  epilogue: thread r normalises output row r out of TMEM and stores it, off the softmax warps' path
+//   warp 8      TMA producer: Q tile (double-buffered) and a ring of 32 KB K / V tiles (128 keys x 128 dims, bf16,
 //               128-byte swizzle), one mbarrier per ring slot
-//   warp 1      MMA issuer: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM) and
+//   warp 9      MMA issuer: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM) and
 //               O += P V (P read from TMEM, V as an MN-major shared-memory operand); owns the TMEM allocation
-//   warps 2..5  softmax: thread r owns query row r (= TMEM lane r): loads its S row, applies the ancestor mask
+//   warps 4..7  softmax: thread r owns query row r (= TMEM lane r): loads its S row, applies the ancestor mask
 //               (a 128-bit mask kept in registers, shifted to the tile), exp2 with a lazily updated reference
 //               maximum, writes P (bf16) over S in TMEM, rescales O in TMEM only when the maximum moved by
 //               more than 2^8, and finally normalises and stores the output row
@@ -18,6 +19,25 @@
 
 #include "tr_internal.cuh"
 
+// Optional timeline instrumentation (off in normal builds): with -DTR_TC_STAMPS=<cta+1> the chosen CTA records
+// SM-clock stamps of a few events per unit, read back with tr_debug_stamps().
+#ifndef TR_TC_STAMPS
+#define TR_TC_STAMPS 0
+#endif
+#if TR_TC_STAMPS
+__device__ long long g_stamps[4 * 16 * 8];
+#define WAITACC(k, expr) { const long long w0__ = clock64(); expr; if (blockIdx.x == TR_TC_STAMPS - 1) g_stamps[(0 * 16 + 15) * 8 + (k)] += clock64() - w0__; }
+#define USTAMP(role, unit, k) \
+  { if (blockIdx.x == TR_TC_STAMPS - 1 && (unit) < 16) g_stamps[((role) * 16 + (unit)) * 8 + (k)] = clock64(); }
+extern "C" int tr_debug_stamps(long long* host) {
+  cudaDeviceSynchronize();
+  return static_cast<int>(cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 4 * 16 * 8));
+}
+#else
+#define USTAMP(role, unit, k) {}
+#define WAITACC(k, expr) { expr; }
+#endif
+
 namespace {
 
 constexpr int BK = 128;          // keys per tile
@@ -25,7 +45,10 @@ constexpr int HD = 128;          // head_dim
 constexpr int NST = 5;           // ring slots (K and V tiles alternate)
 constexpr int TILE_BYTES = BK * HD * 2;       // 32 KB
 constexpr int HALF_BYTES = TILE_BYTES / 2;    // one TMA box: 64 dims x 128 rows
-constexpr int NTHREADS = 192;
+constexpr int NTHREADS = 384;       // warps 0-3 epilogue, 4-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle
+constexpr int WARP_PRODUCER = 8, WARP_MMA = 9;
+// Registers are re-balanced per warpgroup after start-up (setmaxnreg): 12 warps are launched at 168 each.
+constexpr int REGS_EPILOGUE = 112, REGS_SOFTMAX = 240, REGS_CONTROL = 96;
 constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about two seconds of SM clock
 
 struct TcParams {
@@ -36,6 +59,7 @@ struct TcParams {
   float* part_ml;
   uint32_t* flags;
   int N, Hq, Hkv, L, S, n_units;
+  uint32_t div_group[2], div_S[2], div_Hkv[2], div_L[2];  // (multiplier, shift) for exact u32 division
   int64_t os_b, os_h, os_t, os_l;
   float scale_log2;
 };
@@ -46,10 +70,14 @@ constexpr int SM_RING = 2 * TILE_BYTES;               // NST x 32 KB
 constexpr int SM_BAR = SM_RING + NST * TILE_BYTES;    // mbarriers
 constexpr int BAR_FULL = 0, BAR_EMPTY = NST, BAR_QFULL = 2 * NST, BAR_QEMPTY = BAR_QFULL + 2,
               BAR_SFULL = BAR_QEMPTY + 2, BAR_PFULL = BAR_SFULL + 2, BAR_PVDONE = BAR_PFULL + 2,
-              BAR_OFREE = BAR_PVDONE + 2, BAR_COUNT = BAR_OFREE + 2;
+              BAR_OFREE = BAR_PVDONE + 2, BAR_OREADY = BAR_OFREE + 2, BAR_LFULL = BAR_OREADY + 2,
+              BAR_COUNT = BAR_LFULL + 2;
 constexpr int SM_MISC = SM_BAR + BAR_COUNT * 8;       // tmem base (4 B), abort flag (4 B)
-constexpr int SM_TOTAL = SM_MISC + 16;
-constexpr int SMEM_BYTES = SM_TOTAL + 1024;           // slack for manual 1024-byte alignment
+constexpr int SM_LM = SM_MISC + 16;                   // per O buffer: row sums l[128] and reference maxima m[128]
+constexpr int SM_CTX = SM_LM + 2 * 2 * 128 * 4;        // cached context lengths
+constexpr int SM_TOTAL = SM_CTX + 64 * 4;
+constexpr int SMEM_BYTES = SM_TOTAL;                  // the tiles sit at the 1024-byte aligned start of the window
+static_assert(SMEM_BYTES <= 232448, "exceeds the 227 KB a CTA can opt in to");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -77,7 +105,7 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completes.
 // kBackoff: sleep a little between polls (the single-thread producer / MMA roles share their scheduler with a
 // softmax warp and should not take its issue slots).
-template <bool kBackoff = true>
+template <bool kBackoff = false>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
@@ -182,22 +210,59 @@ struct Unit {
   int t0, t1, C;
 };
 
-__device__ __forceinline__ Unit decode_unit(const TcParams& p, int u) {
+// u / d for 0 <= u < 2^31 with a host-computed (multiplier, shift): no hardware divide in the single-thread roles.
+__device__ __forceinline__ uint32_t fast_div(uint32_t u, const uint32_t (&ms)[2]) {
+  return static_cast<uint32_t>((static_cast<uint64_t>(u) * ms[0]) >> ms[1]);
+}
+
+constexpr int CTX_CACHE = 64;  // context lengths of the first 64 sequences are staged in shared memory
+
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, int u, const int* s_ctx) {
   Unit x;
   x.slot = u;
-  const int group = p.Hq / p.Hkv;
-  const int gq = u % group; u /= group;
-  x.split = u % p.S; u /= p.S;
-  x.kvh = u % p.Hkv; u /= p.Hkv;
-  x.layer = u % p.L; u /= p.L;
-  x.b = u;
-  x.h = x.kvh * group + gq;
-  x.C = p.ctx_len[x.b];
+  const uint32_t group = static_cast<uint32_t>(p.Hq / p.Hkv);  // (one divide, by values fixed for the launch)
+  uint32_t v = static_cast<uint32_t>(u), q;
+  q = fast_div(v, p.div_group); const uint32_t gq = v - q * group; v = q;
+  q = fast_div(v, p.div_S); x.split = static_cast<int>(v - q * p.S); v = q;
+  q = fast_div(v, p.div_Hkv); x.kvh = static_cast<int>(v - q * p.Hkv); v = q;
+  q = fast_div(v, p.div_L); x.layer = static_cast<int>(v - q * p.L); v = q;
+  x.b = static_cast<int>(v);
+  x.h = x.kvh * static_cast<int>(group) + static_cast<int>(gq);
+  x.C = x.b < CTX_CACHE ? s_ctx[x.b] : p.ctx_len[x.b];
   const int T = (x.C + p.N + BK - 1) / BK;
   x.t0 = static_cast<int>(static_cast<int64_t>(T) * x.split / p.S);
   x.t1 = static_cast<int>(static_cast<int64_t>(T) * (x.split + 1) / p.S);
   return x;
 }
+
+// Walks this CTA's tiles in order: units blockIdx.x, blockIdx.x + gridDim.x, ... (empty units skipped), tiles
+// t0..t1-1 inside each.  `ui` numbers the non-empty units, `g` the tiles, both from 0.
+struct TileCursor {
+  Unit x;
+  int u, j, nt;
+  uint32_t ui, g;
+  bool valid;
+  __device__ __forceinline__ void seek(const TcParams& p, const int* s_ctx) {
+    while (u < p.n_units) {
+      x = decode_unit(p, u, s_ctx);
+      nt = x.t1 - x.t0;
+      if (nt > 0) { j = 0; valid = true; return; }
+      u += gridDim.x;
+    }
+    valid = false;
+  }
+  __device__ __forceinline__ void init(const TcParams& p, const int* s_ctx) {
+    u = blockIdx.x; ui = 0; g = 0; j = 0; nt = 0;
+    seek(p, s_ctx);
+  }
+  __device__ __forceinline__ void next(const TcParams& p, const int* s_ctx) {
+    ++g;
+    if (++j < nt) return;
+    u += gridDim.x;
+    ++ui;
+    seek(p, s_ctx);
+  }
+};
 
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
@@ -208,16 +273,24 @@ __device__ __forceinline__ float fast_exp2(float x) {
 __global__ void __launch_bounds__(NTHREADS, 1)
 tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const TcParams p) {
-  extern __shared__ unsigned char smem_raw[];
-  const uint32_t raw = smem_u32(smem_raw);
-  const uint32_t base = (raw + 1023u) & ~1023u;
-  unsigned char* base_ptr = smem_raw + (base - raw);
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const uint32_t base = smem_u32(smem_raw);
+  unsigned char* base_ptr = smem_raw;
+  if (base & 1023u) {  // swizzled tiles need a 1024-byte aligned window; not expected, but checked
+    if (threadIdx.x == 0) atomicOr(p.flags, TR_FLAG_WAIT_TIMEOUT);
+    return;
+  }
   const uint32_t bars = base + SM_BAR;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(base_ptr + SM_MISC);
   volatile uint32_t* s_abort = s_tmem + 1;
   auto bar = [&](int i) { return bars + static_cast<uint32_t>(i) * 8u; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int* s_ctx = reinterpret_cast<int*>(base_ptr + SM_CTX);
+  {
+    const int nb = p.n_units / (p.L * p.Hq * p.S);  // sequences
+    if (tid >= 64 && tid - 64 < CTX_CACHE && tid - 64 < nb) s_ctx[tid - 64] = p.ctx_len[tid - 64];
+  }
 
   if (tid == 0) {
     for (int i = 0; i < NST; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
@@ -228,12 +301,14 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(bar(BAR_PFULL + i), 128);
       mbar_init(bar(BAR_PVDONE + i), 1);
       mbar_init(bar(BAR_OFREE + i), 128);
+      mbar_init(bar(BAR_OREADY + i), 1);
+      mbar_init(bar(BAR_LFULL + i), 128);
     }
     *s_abort = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
-  if (warp == 1) {  // TMEM: all 512 columns (one CTA per SM)
+  if (warp == WARP_MMA) {  // TMEM: all 512 columns (one CTA per SM)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + SM_MISC), "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -242,17 +317,22 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  float* s_lm = reinterpret_cast<float*>(base_ptr + SM_LM);  // [2 O buffers][l: 128 | m: 128]
 
-  if (warp == 0) {
+  // Each warpgroup first re-sizes its register budget: the light roles hand registers to the softmax warps.
+  if (warp >= 8) {
+  asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_CONTROL));
+  if (warp == WARP_PRODUCER) {
     // =========================== TMA producer ===========================
     if (lane == 0) {
       uint32_t ui = 0, c = 0;  // non-empty units done by this CTA; ring entries issued
       bool ok = true;
       const uint64_t pol = l2_policy_evict_first();
       for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
-        const Unit x = decode_unit(p, u);
+        const Unit x = decode_unit(p, u, s_ctx);
         if (x.t0 >= x.t1) continue;
         const uint32_t qb = ui & 1u;
+        USTAMP(0, ui, 0)
         ok = mbar_wait(bar(BAR_QEMPTY + qb), ((ui >> 1) & 1u) ^ 1u, s_abort);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_QFULL + qb), TILE_BYTES);
@@ -262,7 +342,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = c % NST, par = ((c / NST) & 1u) ^ 1u;
-            ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort);
+            WAITACC(0, ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort))
             if (!ok) break;
             const CUtensorMap* m = kv == 0 ? &map_k : &map_v;
             const uint32_t dst = base + SM_RING + slot * TILE_BYTES;
@@ -271,25 +351,35 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tma_load_5d_hint(dst + HALF_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b, pol);
             ++c;
           }
+          if (t == x.t0) USTAMP(0, ui, 1)
         }
+        USTAMP(0, ui, 2)
         ++ui;
       }
     }
     __syncwarp();
-  } else if (warp == 1) {
+  } else if (warp == WARP_MMA) {
     // =========================== MMA issuer ===========================
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = make_idesc(false);
       constexpr uint32_t IDESC_PV = make_idesc(true);
-      uint32_t ui = 0, c = 0, g = 0;  // units, ring entries consumed, tiles (S buffers) issued
+      // One flat stream of tiles over all of this CTA's units.  Tile g uses S/P buffer g&1 and ring entries 2g (K)
+      // and 2g+1 (V).  The QK of tile g+1 is issued before the PV of tile g - also across a unit boundary, so the
+      // first scores of the next unit are ready when the softmax warps finish the current one.
       bool ok = true;
-      // software pipeline over tiles: QK(j+1) is issued before PV(j)
-      auto issue_qk = [&](uint32_t qb, uint32_t gg) -> bool {
-        const uint32_t sb = gg & 1u;
-        // the S/P buffer is free once PV of tile gg-2 has completed
-        if (!mbar_wait(bar(BAR_PVDONE + sb), ((gg >> 1) & 1u) ^ 1u, s_abort)) return false;
-        const uint32_t slot = c % NST;
-        if (!mbar_wait(bar(BAR_FULL + slot), (c / NST) & 1u, s_abort)) return false;
+      TileCursor kc, vc;
+      kc.init(p, s_ctx);
+      vc.init(p, s_ctx);
+      auto issue_qk = [&]() -> bool {  // S = Q K^T of the tile under kc
+        const uint32_t sb = kc.g & 1u, c = 2u * kc.g, slot = c % NST, qb = kc.ui & 1u;
+        bool w = true;
+        if (kc.j == 0) WAITACC(4, w = mbar_wait(bar(BAR_QFULL + qb), (kc.ui >> 1) & 1u, s_abort))
+        if (!w) return false;
+        // the S/P buffer is free once the PV of tile g-2 has completed
+        WAITACC(3, w = mbar_wait(bar(BAR_PVDONE + sb), ((kc.g >> 1) & 1u) ^ 1u, s_abort))
+        if (!w) return false;
+        WAITACC(1, w = mbar_wait(bar(BAR_FULL + slot), (c / NST) & 1u, s_abort))
+        if (!w) return false;
         tc_fence_after();
         const uint32_t qa = base + SM_Q + qb * TILE_BYTES, ka = base + SM_RING + slot * TILE_BYTES;
 #pragma unroll
@@ -297,56 +387,50 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
           tc_mma_ss(tmem + sb * 128u, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK, k > 0);
         }
-        tc_commit(bar(BAR_EMPTY + slot));   // K tile consumed
-        tc_commit(bar(BAR_SFULL + sb));     // S ready for the softmax warps
-        ++c;
+        tc_commit(bar(BAR_EMPTY + slot));                          // K tile consumed
+        tc_commit(bar(BAR_SFULL + sb));                            // S ready for the softmax warps
+        if (kc.j == kc.nt - 1) tc_commit(bar(BAR_QEMPTY + qb));    // unit's last QK: Q buffer free when it finishes
+        if (kc.j == 0) USTAMP(1, kc.ui, 0)
+        kc.next(p, s_ctx);
         return true;
       };
-      for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
-        const Unit x = decode_unit(p, u);
-        const int nt = x.t1 - x.t0;
-        if (nt <= 0) continue;
-        const uint32_t qb = ui & 1u, ob = ui & 1u;
-        ok = mbar_wait(bar(BAR_QFULL + qb), (ui >> 1) & 1u, s_abort);
-        if (!ok) break;
-        ok = issue_qk(qb, g);
-        for (int j = 0; j < nt && ok; ++j) {
-          // ring order is K0 V0 K1 V1 ...: V(j) sits at entry c, K(j+1) at entry c+1; the QK of tile j+1 goes
-          // first so that it overlaps the softmax of tile j
-          const uint32_t vslot = c % NST, vpar = (c / NST) & 1u;
-          ++c;
-          if (j + 1 < nt) {
-            ok = issue_qk(qb, g + 1);
-            if (!ok) break;
-          } else {
-            tc_commit(bar(BAR_QEMPTY + qb));  // all QK of this unit issued: Q buffer free when they finish
-          }
-          if (j == 0) {  // the O buffer must have been drained by the epilogue of unit ui-2
-            ok = mbar_wait(bar(BAR_OFREE + ob), ((ui >> 1) & 1u) ^ 1u, s_abort);
-            if (!ok) break;
-          }
-          const uint32_t sb = g & 1u;
-          ok = mbar_wait(bar(BAR_PFULL + sb), (g >> 1) & 1u, s_abort) && mbar_wait(bar(BAR_FULL + vslot), vpar, s_abort);
+      if (kc.valid) ok = issue_qk();
+      while (ok && vc.valid) {
+        if (kc.valid) {
+          ok = issue_qk();
           if (!ok) break;
-          tc_fence_after();
-          const uint32_t va = base + SM_RING + vslot * TILE_BYTES;
-#pragma unroll
-          for (int k = 0; k < BK / 16; ++k) {
-            // A = P (bf16 pairs, 8 TMEM columns per 16 keys); B = V tile, MN-major: 64-dim chunks 16 KB apart,
-            // 8-key groups 1 KB apart, 16 keys per step = 2 KB
-            tc_mma_ts(tmem + 256u + ob * 128u, tmem + sb * 128u + k * 8u, smem_desc(va + k * 2048, HALF_BYTES, 1024),
-                      IDESC_PV, (j > 0 || k > 0) ? 1u : 0u);
-          }
-          tc_commit(bar(BAR_EMPTY + vslot));  // V tile consumed
-          tc_commit(bar(BAR_PVDONE + sb));    // P consumed, O updated
-          ++g;
         }
-        ++ui;
+        const uint32_t sb = vc.g & 1u, ob = vc.ui & 1u, c = 2u * vc.g + 1u, vslot = c % NST;
+        if (vc.j == 0) {  // the O buffer must have been drained by the epilogue of unit ui-2
+          ok = mbar_wait(bar(BAR_OFREE + ob), ((vc.ui >> 1) & 1u) ^ 1u, s_abort);
+          if (!ok) break;
+        }
+        WAITACC(2, ok = mbar_wait(bar(BAR_PFULL + sb), (vc.g >> 1) & 1u, s_abort))
+        if (!ok) break;
+        WAITACC(5, ok = mbar_wait(bar(BAR_FULL + vslot), (c / NST) & 1u, s_abort))
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t va = base + SM_RING + vslot * TILE_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / 16; ++k) {
+          // A = P (bf16 pairs, 8 TMEM columns per 16 keys); B = V tile, MN-major: 64-dim chunks 16 KB apart,
+          // 8-key groups 1 KB apart, 16 keys per step = 2 KB
+          tc_mma_ts(tmem + 256u + ob * 128u, tmem + sb * 128u + k * 8u, smem_desc(va + k * 2048, HALF_BYTES, 1024),
+                    IDESC_PV, (vc.j > 0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit(bar(BAR_EMPTY + vslot));                             // V tile consumed
+        tc_commit(bar(BAR_PVDONE + sb));                               // P consumed, O updated
+        if (vc.j == vc.nt - 1) tc_commit(bar(BAR_OREADY + ob));        // the unit's output is complete
+        if (vc.j == 0) USTAMP(1, vc.ui, 1)
+        if (vc.j == vc.nt - 1) USTAMP(1, vc.ui, 2)
+        vc.next(p, s_ctx);
       }
     }
     __syncwarp();
-  } else {
-    // =========================== softmax / correction / epilogue ===========================
+  }
+  } else if (warp >= 4) {
+    // =========================== softmax / correction ===========================
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(REGS_SOFTMAX));
     const int r = (warp & 3) * 32 + lane;                 // query row == TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     uint32_t anc[4];
@@ -355,7 +439,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     uint32_t ui = 0, g = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
-      const Unit x = decode_unit(p, u);
+      const Unit x = decode_unit(p, u, s_ctx);
       const int nt = x.t1 - x.t0;
       float m_ref = -INFINITY, l = 0.f;
       const uint32_t ob = ui & 1u;
@@ -365,6 +449,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
         if (!ok) break;
         tc_fence_after();
+        if (tid == 128 && j == 0) USTAMP(2, ui, 0)
         uint32_t sreg[4][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q) tc_ld32(tmem + lane_base + sb * 128u + q * 32u, sreg[q]);
@@ -460,9 +545,35 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar(BAR_PFULL + sb));
+        if (tid == 128 && j == 0) USTAMP(2, ui, 1)
+        if (tid == 128 && j == nt - 1) USTAMP(2, ui, 2)
       }
       if (!ok) break;
-      // ---- epilogue of the unit
+      if (nt <= 0) continue;  // empty split: the epilogue warps write its (empty) partial
+      // ---- hand the unit to the epilogue warps: row sum and reference maximum go through shared memory.  The
+      //      slot was last read by the epilogue of unit ui-2, which signalled OFREE when it was done with it.
+      ok = mbar_wait<false>(bar(BAR_OFREE + ob), ((ui >> 1) & 1u) ^ 1u, s_abort);
+      ok = __all_sync(0xFFFFFFFFu, ok);
+      if (!ok) break;
+      s_lm[ob * 256 + r] = l;
+      s_lm[ob * 256 + 128 + r] = m_ref;
+      mbar_arrive(bar(BAR_LFULL + ob));
+      if (tid == 128) USTAMP(2, ui, 3)
+      ++ui;
+    }
+  } else {
+    // =========================== epilogue ===========================
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(REGS_EPILOGUE));
+    // Thread r owns output row r: waits until the unit's last PV has landed (OREADY) and the softmax warps have
+    // published the row sums (LFULL), then normalises O out of TMEM and stores it (bf16 rows, or the fp32
+    // partial of a KV split), so the softmax warps never stop at a unit boundary.
+    const int r = warp * 32 + lane;
+    const uint32_t lane_base = static_cast<uint32_t>(warp * 32) << 16;
+    uint32_t ui = 0;
+    bool ok = true;
+    for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
+      const Unit x = decode_unit(p, u, s_ctx);
+      const int nt = x.t1 - x.t0;
       float* po = p.part_o + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 128;
       float* pml = p.part_ml + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 2;
       if (nt <= 0) {  // empty split: contributes nothing
@@ -472,11 +583,13 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         continue;
       }
-      const uint32_t lb = (g - 1u) & 1u;
-      ok = mbar_wait<false>(bar(BAR_PVDONE + lb), ((g - 1u) >> 1) & 1u, s_abort);
+      const uint32_t ob = ui & 1u, par = (ui >> 1) & 1u;
+      ok = mbar_wait<false>(bar(BAR_LFULL + ob), par, s_abort) && mbar_wait<false>(bar(BAR_OREADY + ob), par, s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
+      if (tid == 0) USTAMP(3, ui, 0)
+      const float l = s_lm[ob * 256 + r], m_ref = s_lm[ob * 256 + 128 + r];
       const float inv = 1.f / l;
       __nv_bfloat16* orow = p.out + x.b * p.os_b + x.layer * p.os_l + x.h * p.os_h + static_cast<int64_t>(r) * p.os_t;
 #pragma unroll
@@ -484,7 +597,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         uint32_t oreg[32];
         tc_ld32(tmem + lane_base + 256u + ob * 128u + q * 32u, oreg);
         tc_wait_ld();
-        if (q == 3) {  // the O buffer is in registers: hand it back to the MMA warp
+        if (q == 3) {  // O (and l, m) are in registers: hand the buffer back to the MMA and softmax warps
           tc_fence_before();
           mbar_arrive(bar(BAR_OFREE + ob));
         }
@@ -514,6 +627,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         pml[0] = m_ref;
         pml[1] = l;
       }
+      if (tid == 0) USTAMP(3, ui, 1)
       ++ui;
     }
   }
@@ -526,7 +640,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     for (int i = 0; i < 200; ++i) __nanosleep(1000);
     __syncthreads();
   }
-  if (warp == 1) {
+  if (warp == WARP_MMA) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
   }
@@ -573,6 +687,15 @@ tr_status tr_attention_tc_setup() {
 
 void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
 
+// (M, k) with floor(u / d) == (u * M) >> k for all 0 <= u < 2^31: k = 31 + ceil(log2 d), M = ceil(2^k / d) < 2^32.
+static void magic_u32(uint32_t d, uint32_t (&ms)[2]) {
+  uint32_t l = 0;
+  while ((1ull << l) < d) ++l;
+  const uint32_t k = 31 + l;
+  ms[0] = static_cast<uint32_t>(((1ull << k) + d - 1) / d);
+  ms[1] = k;
+}
+
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s) {
   if (a->head_dim != HD) return TR_ERR_UNSUPPORTED;
   const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * a->n_q_heads;
@@ -590,6 +713,10 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   p.scale_log2 = scale * 1.4426950408889634f;
   p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK);
   p.n_units = static_cast<int>(base * p.S);
+  magic_u32(static_cast<uint32_t>(a->n_q_heads / a->n_kv_heads), p.div_group);
+  magic_u32(static_cast<uint32_t>(p.S), p.div_S);
+  magic_u32(static_cast<uint32_t>(p.Hkv), p.div_Hkv);
+  magic_u32(static_cast<uint32_t>(p.L), p.div_L);
 
   // Q is addressed as (dim, head, node, layer, sequence): in the usual [.., node, head, dim] layout the head
   // stride is the smaller one, and the tile (64 dims x 1 head x 128 nodes) lands in shared memory as 128 rows.

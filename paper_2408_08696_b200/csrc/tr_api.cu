@@ -301,3 +301,11 @@ extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_s
   TR_CUDA_TRY(cudaStreamSynchronize(s));
   return TR_OK;
 }
+
+// Debugging aid (not part of the public header): copies the first n floats of the split-KV scratch to the host.
+extern "C" tr_status tr_debug_read_scratch(tr_ctx* ctx, float* host, int32_t n) {
+  if (!ctx || !host || n < 0) return TR_ERR_INVALID_ARG;
+  TR_CUDA_TRY(cudaDeviceSynchronize());
+  TR_CUDA_TRY(cudaMemcpy(host, ctx->d_attn_part_o, sizeof(float) * n, cudaMemcpyDeviceToHost));
+  return TR_OK;
+}
