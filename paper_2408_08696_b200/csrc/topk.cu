@@ -39,6 +39,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   __shared__ u64 s_cand[TOPK_CAND_CAP];
   __shared__ u64 s_out[TR_MAX_K];
   __shared__ u64 s_merge[TOPK_MERGE_CAP];
+  __shared__ u64 s_tau;
   __shared__ int s_cnt;
   __shared__ int s_last;
 
@@ -91,26 +92,30 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
     if ((lane & 15) == 0) s_gmax[tid >> 4] = (static_cast<u64>(mh) << 32) | ml;
   }
   __syncthreads();
-  // rank by counting, done by every warp for itself: the group maximum that has exactly k-1 larger ones is the
+  // rank by counting, by half a warp for the whole CTA: the group maximum that has exactly k-1 larger ones is the
   // threshold; with fewer than k non-empty groups the threshold is 0 and every key is a candidate
-  u64 tau;
-  {
+  if (warp == 0) {
     const u64 mine = lane < G ? s_gmax[lane] : 0ull;
     int larger = 0;
 #pragma unroll
     for (int i = 0; i < G; ++i) larger += (s_gmax[i] > mine) ? 1 : 0;
     const unsigned hit = __ballot_sync(0xFFFFFFFFu, lane < G && mine != 0ull && larger == k - 1);
-    const int src = hit ? (__ffs(hit) - 1) : 0;
-    const uint32_t th = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(mine >> 32), src);
-    const uint32_t tl = __shfl_sync(0xFFFFFFFFu, static_cast<uint32_t>(mine), src);
-    tau = hit ? ((static_cast<u64>(th) << 32) | tl) : 0ull;
+    if (hit == 0u) {
+      if (lane == 0) s_tau = 0ull;
+    } else if (lane == __ffs(hit) - 1) {
+      s_tau = mine;
+    }
   }
+  __syncthreads();
+  const u64 tau = s_tau;
   // ---- (3) candidates: only threads whose own maximum reaches the threshold look at their values
   if (tmax != 0 && tmax >= tau) {
+    const uint32_t tau_hi = static_cast<uint32_t>(tau >> 32);
 #pragma unroll
     for (int j = 0; j < E; ++j) {
       const int i = index_of(j);
-      if (i < V) {
+      // cheap filter on the value alone, then the exact (value, index) comparison
+      if (i < V && static_cast<uint32_t>(topk_key(v[j], 0u) >> 32) >= tau_hi) {
         const u64 key = topk_key(v[j], i);
         if (key >= tau) {
           const int p = atomicAdd(&s_cnt, 1);
@@ -129,15 +134,10 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
       const u64 mine = s_cand[t];
       int larger = 0;
       for (int i = 0; i < cnt; ++i) larger += (s_cand[i] > mine) ? 1 : 0;
-      if (larger < k) {
-        my_part[larger] = mine;
-        __threadfence();  // published device-wide before this CTA takes its ticket
-      }
+      if (larger < k) my_part[larger] = mine;
     }
-    if (tid >= cnt && tid < k) {
-      my_part[tid] = 0ull;
-      __threadfence();
-    }
+    if (tid >= cnt && tid < k) my_part[tid] = 0ull;
+    // (these writes are published by the barrier below together with thread 0's fence, which is cumulative)
   } else {
     // More candidates than the buffer holds (only with massive ties or adversarial layouts): select straight
     // from the registers, round by round, the whole CTA taking part.
