@@ -315,7 +315,11 @@ def run_ours(args, w):
 
 
 # DRAM bytes (read + write) of one attention launch from the committed ncu capture (see profiles/), per workload.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/tr_attn_tc_kernel_llama2-7b_16layers.md: (300.07 MB read + 3.85 MB written) per 16-layer launch,
+    # scaled to the 32 layers of one benchmark launch (traffic is proportional to the layers processed)
+    "llama2-7b": 2 * (300_069_376 + 3_845_888),
+}
 
 
 def main():
