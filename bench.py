@@ -195,7 +195,6 @@ def run_ours(args, w):
     torch.cuda.synchronize()
     sampler = ClockSampler(local_rank) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_new_sum = 0
     e0.record(stream)
     for i in range(K):
         graphs[(W + i) % dw.n_rot].replay()
@@ -205,8 +204,12 @@ def run_ours(args, w):
     elapsed_ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if sampler else None
     agg = replicas.aggregate(elapsed_ms, K, device=dev if world > 1 else "cpu")
-    n_new_sum = int(dw.out["n_new"].sum().item())
     flags = tr.tr_device_flags(dw.ctx)
+    # acceptance statistic of the toy model (a sanity figure, not a result): 64 untimed steps, n_new read each step
+    n_new_sum, n_stat = 0, 64
+    for i in range(n_stat):
+        graphs[(W + K + i) % dw.n_rot].replay()
+        n_new_sum += int(dw.out["n_new"].sum().item())
 
     # ---- dominant kernel (tree attention) alone: event pair around every launch, same stream
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
@@ -305,7 +308,7 @@ def run_ours(args, w):
                     "steps": Ke},
             "gpu_launches": dw.kernels_per_step() * K,
             "clocks": clocks,
-            "new_tokens_last_step": n_new_sum / B,
+            "mean_new_tokens_per_step": n_new_sum / (B * n_stat),
             "device_flags": flags,
         }
         print(json.dumps(line), flush=True)

@@ -265,8 +265,12 @@ __global__ void __launch_bounds__(256) tr_attn_mma_kernel(const AttnParams p) {
 }
 
 // Merge the per-split partial softmaxes: out = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s.
-__global__ void tr_attn_combine_kernel(const AttnParams p, int D) {
-  const int row = blockIdx.x;   // tree node
+// One CTA per (8 tree nodes, query-head unit): 32 lanes x float4 cover the 128 (or 64) dims of a row.
+constexpr int COMBINE_ROWS = 8;
+__global__ void __launch_bounds__(COMBINE_ROWS * 32) tr_attn_combine_kernel(const AttnParams p, int D) {
+  const int row = blockIdx.x * COMBINE_ROWS + (threadIdx.x >> 5);  // tree node
+  const int d = (threadIdx.x & 31) * 4;
+  if (row >= p.N || d >= D) return;
   int u = blockIdx.y;           // (b, layer, kv head, q-in-group)
   const int group = p.Hq / p.Hkv;
   const int gq = u % group;
@@ -275,33 +279,44 @@ __global__ void tr_attn_combine_kernel(const AttnParams p, int D) {
   const int layer = (blg / p.Hkv) % p.L;
   const int b = blg / (p.Hkv * p.L);
   const int h = kvh * group + gq;
-  const int d = threadIdx.x;
   float mstar = -INFINITY;
   for (int s = 0; s < p.S; ++s) {
     const size_t slot = (static_cast<size_t>(blg) * p.S + s) * group + gq;
     mstar = fmaxf(mstar, p.part_ml[(slot * ATTN_PART_ROWS + row) * 2]);
   }
-  float acc = 0.f, den = 0.f;
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float den = 0.f;
   for (int s = 0; s < p.S; ++s) {
     const size_t slot = (static_cast<size_t>(blg) * p.S + s) * group + gq;
-    const float m = p.part_ml[(slot * ATTN_PART_ROWS + row) * 2];
-    const float l = p.part_ml[(slot * ATTN_PART_ROWS + row) * 2 + 1];
-    const float w = (m == -INFINITY) ? 0.f : exp2f(m - mstar);
-    acc += w * p.part_o[(slot * ATTN_PART_ROWS + row) * 128 + d];
-    den += w * l;
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (slot * ATTN_PART_ROWS + row) * 2);
+    const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mstar);
+    const float4 o = *reinterpret_cast<const float4*>(p.part_o + (slot * ATTN_PART_ROWS + row) * 128 + d);
+    acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+    den += w * ml.y;
   }
-  __nv_bfloat16* op = p.out + b * p.os_b + layer * p.os_l + h * p.os_h + row * p.os_t;
-  op[d] = __float2bfloat16_rn(acc / den);
+  const float inv = 1.f / den;
+  __nv_bfloat16* op = p.out + b * p.os_b + layer * p.os_l + h * p.os_h + row * p.os_t + d;
+  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  uint2 w2;
+  w2.x = *reinterpret_cast<uint32_t*>(&lo);
+  w2.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(op) = w2;
 }
 
 }  // namespace
 
-int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys) {
+// `fill_once`: the caller is a persistent one-CTA-per-SM kernel, so the split count is chosen to give every SM at
+// most one unit (no second, partly filled round); otherwise about two CTAs' worth of units per SM.
+int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys, bool fill_once) {
   const int tiles = (a->max_ctx + ctx->n_nodes + tile_keys - 1) / tile_keys;
   int S = a->splits;
   if (S <= 0) {
-    const int want = 2 * ctx->sm_count;
-    S = base_units >= want ? 1 : (want + base_units - 1) / base_units;
+    if (fill_once) {
+      S = base_units >= ctx->sm_count ? 1 : ctx->sm_count / base_units;
+    } else {
+      const int want = 2 * ctx->sm_count;
+      S = base_units >= want ? 1 : (want + base_units - 1) / base_units;
+    }
     if (S > 16) S = 16;
   }
   if (S > tiles) S = tiles;
@@ -325,7 +340,8 @@ void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cuda
   AttnParams p = make_params(ctx, a);
   p.S = S;
   const unsigned base = static_cast<unsigned>(ctx->batch) * a->n_layers * a->n_q_heads;
-  tr_attn_combine_kernel<<<dim3(ctx->n_nodes, base), a->head_dim, 0, s>>>(p, a->head_dim);
+  tr_attn_combine_kernel<<<dim3((ctx->n_nodes + COMBINE_ROWS - 1) / COMBINE_ROWS, base), COMBINE_ROWS * 32, 0, s>>>(
+      p, a->head_dim);
 }
 
 static AttnParams make_params(tr_ctx* ctx, const tr_attn_args* a) {
@@ -352,7 +368,7 @@ tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream
   AttnParams p = make_params(ctx, a);
   const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * a->n_q_heads;
   if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
-  p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BN);
+  p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BN, false);
   if (p.S > 1 && base * p.S > ATTN_MAX_PART_SLOTS) return TR_ERR_UNSUPPORTED;
   const int nwarps = (ctx->n_nodes + 15) / 16;
   const int D = a->head_dim;

@@ -711,7 +711,7 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   p.os_b = a->o_stride[0]; p.os_h = a->o_stride[1]; p.os_t = a->o_stride[2]; p.os_l = a->layer_stride_o;
   const float scale = a->scale != 0.f ? a->scale : 1.0f / sqrtf(static_cast<float>(a->head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
-  p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK);
+  p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK, true);
   p.n_units = static_cast<int>(base * p.S);
   magic_u32(static_cast<uint32_t>(a->n_q_heads / a->n_kv_heads), p.div_group);
   magic_u32(static_cast<uint32_t>(p.S), p.div_S);

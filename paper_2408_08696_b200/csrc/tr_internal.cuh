@@ -58,4 +58,4 @@ tr_status tr_attention_mma_setup();
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_tc_setup();
 void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
-int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys);
+int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys, bool fill_once);

@@ -89,7 +89,7 @@ class DeviceWorkload:
         if self.attn is not None:
             n += 1
             base = self.w.batch * self.L * self.w.n_q_heads
-            if self.attn.splits != 1 and base < 2 * 148:
+            if self.attn.splits != 1 and base < 148:
                 n += 1  # split-KV combine
         return n
 
