@@ -264,6 +264,33 @@ def test_attention_llama2_7b_full_size_sampled(harness):
     dw.close()
 
 
+@pytest.mark.parametrize("name", ["llama2-13b", "llama3-8b", "llama2-70b-b8"])
+def test_attention_other_workload_shapes_one_layer_sampled(harness, name):
+    """The other workloads' full head counts, group sizes and context lengths (4096; 8192 with 4 query heads per KV
+    head; eight sequences of 1024..4096 with 8 per KV head), one layer each; the oracle checks a seeded sample of
+    (sequence, query head) outputs."""
+    w = synth.WORKLOADS[name]
+    dw = harness.DeviceWorkload(w, n_layers=1)
+    from paper_2408_08696_b200 import binding as tr
+    tr.tr_tree_attention(dw.ctx, dw.attn)
+    torch.cuda.synchronize()
+    assert tr.tr_device_flags(dw.ctx) == 0
+    q, k, v = synth.attention_inputs(w, 1)
+    group = w.n_q_heads // w.n_kv_heads
+    rng = np.random.default_rng(7)
+    for _ in range(12):
+        b, h = int(rng.integers(0, w.batch)), int(rng.integers(0, w.n_q_heads))
+        g, c = h // group, w.ctx[b]
+        ref = orc.tree_attention(synth.bf16_bits_to_f32(q[b, 0, :, h:h + 1]),
+                                 synth.bf16_bits_to_f32(k[b, 0, g:g + 1, : c + w.n_nodes]),
+                                 synth.bf16_bits_to_f32(v[b, 0, g:g + 1, : c + w.n_nodes]), c, dw.parent)
+        got = dw.o[b, 0, :, h].float().cpu().numpy()
+        mx, rel = attention_close(got, ref[:, 0])
+        assert mx <= ATOL and rel <= RTOL, (name, b, h, mx, rel)
+    assert torch.isfinite(dw.o.float()).all()
+    dw.close()
+
+
 # ------------------------------------------------------------------ whole step, host-buffer entry point
 def test_step_host_matches_device_calls(harness, tr):
     import ctypes as C
