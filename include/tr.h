@@ -47,6 +47,7 @@ typedef int32_t tr_status;
 /* Device flag bits (tr_device_flags). */
 #define TR_FLAG_BAD_TOKEN 1u    /* a tree/root token id was outside [0, V): row skipped / id clamped to 0 */
 #define TR_FLAG_WAIT_TIMEOUT 2u /* a bounded wait inside a kernel ran out (should never happen) */
+#define TR_FLAG_CACHE_FULL 4u   /* tr_commit: no room for another tree behind the grown prefix; sequence left as is */
 
 const char* tr_status_string(tr_status s);
 
@@ -145,6 +146,37 @@ typedef struct {
 tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const int32_t* d_tree, const tr_step_out* out,
                            void* stream);
 int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appendix: maximum acceptance length) */
+
+/*
+ * Commit the accepted path (Sec. 5.4: a step ends by "updating the matrix, input tokens, and key-value cache").
+ * Call after tr_verify_update with its outputs.  For every sequence b with n = n_new[b] and accepted nodes
+ * a_0 = 0 (root), a_1, ..., a_{n-1} (acc_nodes[b]):
+ *   K/V : for every layer and KV head, cache row C_b + a_i moves to row C_b + i (i = 1..n-1; the root's row is in
+ *         place), so rows [0, C_b + n) are the new prefix in order;
+ *   text: out_tokens[b][0..n) (the accepted drafts and the extra greedy token) are appended at
+ *         d_tokens[b * token_capacity + n_tokens[b]];
+ *   then C_b += n and n_tokens[b] += n.  ctx_len lives on the device, so a captured graph keeps replaying while
+ *   the prefix grows (tr_tree_attention reads it there).
+ * A sequence for which C_b + n + N > kv_rows or n_tokens[b] + n > token_capacity is left untouched and
+ * TR_FLAG_CACHE_FULL is set.
+ * DEVICE in/out: k_cache, v_cache (bf16, same addressing as tr_tree_attention), d_ctx_len [batch], d_tokens
+ *   [batch, token_capacity] int32, d_n_tokens [batch].  DEVICE in: d_acc_nodes, d_out_tokens [batch, depth_max+1],
+ *   d_n_new [batch] as written by tr_verify_update.
+ * Errors: TR_ERR_INVALID_ARG (NULL, bad sizes / alignment), TR_ERR_UNSUPPORTED (head_dim not a multiple of 8).
+ */
+typedef struct {
+  void* k_cache; /* DEVICE bf16 */
+  void* v_cache; /* DEVICE bf16 */
+  int32_t n_kv_heads, head_dim, n_layers, kv_rows;
+  int64_t kv_stride[3]; /* (sequence, head, token) in elements */
+  int64_t layer_stride_kv;
+  int32_t* d_ctx_len;
+  int32_t* d_tokens;
+  int32_t token_capacity;
+  int32_t* d_n_tokens;
+} tr_commit_args;
+tr_status tr_commit(tr_ctx* ctx, const tr_commit_args* args, const int32_t* d_acc_nodes, const int32_t* d_out_tokens,
+                    const int32_t* d_n_new, void* stream);
 
 /* Copies the sticky flag word to HOST and synchronises the device. */
 tr_status tr_device_flags(tr_ctx* ctx, uint32_t* host_flags);

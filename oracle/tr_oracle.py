@@ -257,3 +257,23 @@ def verify_update(M, S, logits, parent, rank):
     nxt = bfs_tree(M, parent, rank, next_root)
     return dict(topk=O, n_new=n_new, acc_nodes=acc_nodes, out_tokens=out_tokens,
                 next_root=next_root, next_tree=nxt)
+
+
+# --------------------------------------------------------------------------
+# Commit of the accepted path (Sec. 5.4: "updating the matrix, input tokens, and key-value cache")
+# --------------------------------------------------------------------------
+def commit(k, v, ctx_len, tokens, acc_nodes, out_tokens):
+    """After verification the accepted nodes (root first) are the tokens whose keys and values now belong to the
+    prefix: their cache rows are gathered, in path order, right behind the old prefix; the step's new tokens
+    (accepted drafts + the extra greedy token) are appended to the text; the prefix grows by their count.
+
+    k, v : [..., rows, D] caches with the tree's rows at ctx_len .. ctx_len + N - 1 (modified in place)
+    Returns (new ctx_len, new token list).
+    Pinned by: a hand-worked example; the gathered rows equal the rows of the accepted path taken from a copy.
+    """
+    n = len(acc_nodes)
+    src_k = k[..., [ctx_len + a for a in acc_nodes], :].copy()
+    src_v = v[..., [ctx_len + a for a in acc_nodes], :].copy()
+    k[..., ctx_len:ctx_len + n, :] = src_k
+    v[..., ctx_len:ctx_len + n, :] = src_v
+    return ctx_len + n, list(tokens) + [int(t) for t in out_tokens]

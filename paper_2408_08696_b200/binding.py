@@ -26,7 +26,7 @@ lib_synth = C.CDLL(LIB_SYNTH_PATH)
 
 TR_OK = 0
 TR_ERR_INVALID_ARG, TR_ERR_TEMPLATE, TR_ERR_UNSUPPORTED, TR_ERR_CUDA, TR_ERR_NOMEM, TR_ERR_DEVICE_FLAG = -1, -2, -3, -4, -5, -6
-TR_FLAG_BAD_TOKEN, TR_FLAG_WAIT_TIMEOUT = 1, 2
+TR_FLAG_BAD_TOKEN, TR_FLAG_WAIT_TIMEOUT, TR_FLAG_CACHE_FULL = 1, 2, 4
 TR_MAX_NODES, TR_MAX_K = 128, 16
 
 
@@ -53,6 +53,15 @@ class tr_step_out(C.Structure):
                 ("d_topk_idx", "d_n_new", "d_acc_nodes", "d_out_tokens", "d_next_root", "d_next_tree")]
 
 
+class tr_commit_args(C.Structure):
+    _fields_ = [
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p),
+        ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("n_layers", C.c_int32), ("kv_rows", C.c_int32),
+        ("kv_stride", C.c_int64 * 3), ("layer_stride_kv", C.c_int64),
+        ("d_ctx_len", C.c_void_p), ("d_tokens", C.c_void_p), ("token_capacity", C.c_int32), ("d_n_tokens", C.c_void_p),
+    ]
+
+
 class tr_host_io(C.Structure):
     _fields_ = [(n, C.c_void_p) for n in
                 ("h_q", "h_tree_k", "h_tree_v", "h_logits", "h_ctx_len", "d_logits_staging", "d_tree",
@@ -77,6 +86,7 @@ lib.tr_max_new_tokens.argtypes = [C.c_void_p]
 lib.tr_device_flags.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
 lib.tr_step_host.argtypes = [C.c_void_p, C.POINTER(tr_attn_args), C.POINTER(tr_step_out), C.POINTER(tr_host_io),
                              C.c_void_p]
+lib.tr_commit.argtypes = [C.c_void_p, C.POINTER(tr_commit_args), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.tr_topk_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
 lib.tr_topk_noalloc_limits.argtypes = [_P32, _P32]
 lib_synth.trs_patch_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
@@ -229,6 +239,31 @@ def tr_verify_update(ctx, d_logits, d_tree, out_struct, stream=None):
     _check(lib.tr_verify_update(ctx.handle, _dev(d_logits, torch.float32, "d_logits"),
                                 _dev(d_tree, torch.int32, "d_tree"), C.byref(out_struct), _stream(stream)),
            "tr_verify_update")
+
+
+def make_commit_args(ctx, k_cache, v_cache, d_ctx_len, d_tokens, d_n_tokens):
+    """k_cache/v_cache: bf16 [B, L, Hkv, R, D]; d_ctx_len, d_n_tokens int32 [B]; d_tokens int32 [B, capacity]."""
+    a = tr_commit_args()
+    a.k_cache, a.v_cache = _dev(k_cache, torch.bfloat16, "k_cache"), _dev(v_cache, torch.bfloat16, "v_cache")
+    B, L, Hkv, R, D = k_cache.shape
+    if v_cache.shape != k_cache.shape or v_cache.stride() != k_cache.stride() or k_cache.stride(4) != 1:
+        raise ValueError("unsupported cache layout")
+    if B != ctx.batch or tuple(d_tokens.shape[:1]) != (B,) or not d_tokens.is_contiguous():
+        raise ValueError("batch differs from the context")
+    a.n_kv_heads, a.head_dim, a.n_layers, a.kv_rows = Hkv, D, L, R
+    a.kv_stride = (C.c_int64 * 3)(k_cache.stride(0), k_cache.stride(2), k_cache.stride(3))
+    a.layer_stride_kv = k_cache.stride(1)
+    a.d_ctx_len = _dev(d_ctx_len, torch.int32, "d_ctx_len")
+    a.d_tokens = _dev(d_tokens, torch.int32, "d_tokens")
+    a.token_capacity = d_tokens.shape[1]
+    a.d_n_tokens = _dev(d_n_tokens, torch.int32, "d_n_tokens")
+    return a
+
+
+def tr_commit(ctx, args, d_acc_nodes, d_out_tokens, d_n_new, stream=None):
+    _check(lib.tr_commit(ctx.handle, C.byref(args), _dev(d_acc_nodes, torch.int32, "d_acc_nodes"),
+                         _dev(d_out_tokens, torch.int32, "d_out_tokens"), _dev(d_n_new, torch.int32, "d_n_new"),
+                         _stream(stream)), "tr_commit")
 
 
 def tr_device_flags(ctx):

@@ -60,6 +60,7 @@ static tr_status free_all(tr_ctx* c) {
   cudaFree(c->d_M);
   cudaFree(c->d_topk_part);
   cudaFree(c->d_topk_ticket);
+  cudaFree(c->d_seq_ticket);
   cudaFree(c->d_attn_part_o);
   cudaFree(c->d_attn_part_ml);
   cudaFree(c->d_flags);
@@ -138,6 +139,8 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaMalloc(&c->d_topk_part, sizeof(unsigned long long) * rows * c->topk_segs * k));
   TR_INIT_TRY(cudaMalloc(&c->d_topk_ticket, sizeof(unsigned int) * rows));
   TR_INIT_TRY(cudaMemset(c->d_topk_ticket, 0, sizeof(unsigned int) * rows));
+  TR_INIT_TRY(cudaMalloc(&c->d_seq_ticket, sizeof(unsigned int) * batch));
+  TR_INIT_TRY(cudaMemset(c->d_seq_ticket, 0, sizeof(unsigned int) * batch));
 
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_o, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 128));
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_ml, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 2));
@@ -248,6 +251,23 @@ extern "C" tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* a, void*
   // head_dim 128 runs on the tcgen05 / TMA kernel; head_dim 64 on the warp-level MMA kernel
   if (a->head_dim == 128 && !ctx->force_mma) return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
   return tr_launch_attention_mma(ctx, a, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" tr_status tr_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,
+                               const int32_t* d_out_tokens, const int32_t* d_n_new, void* stream) {
+  if (!ctx || !a || !a->k_cache || !a->v_cache || !a->d_ctx_len || !a->d_tokens || !a->d_n_tokens || !d_acc_nodes ||
+      !d_out_tokens || !d_n_new)
+    return TR_ERR_INVALID_ARG;
+  if (a->n_kv_heads < 1 || a->n_layers < 1 || a->kv_rows < ctx->n_nodes || a->token_capacity < 1)
+    return TR_ERR_INVALID_ARG;
+  if (a->head_dim < 8 || a->head_dim % 8 != 0 || a->head_dim > 256) return TR_ERR_UNSUPPORTED;
+  if ((reinterpret_cast<uintptr_t>(a->k_cache) & 15) || (reinterpret_cast<uintptr_t>(a->v_cache) & 15))
+    return TR_ERR_INVALID_ARG;
+  const int64_t strides[4] = {a->kv_stride[0], a->kv_stride[1], a->kv_stride[2], a->layer_stride_kv};
+  for (int64_t s : strides)
+    if (s < 0 || (s & 7)) return TR_ERR_INVALID_ARG;
+  if (a->kv_stride[2] < a->head_dim) return TR_ERR_INVALID_ARG;
+  return tr_launch_commit(ctx, a, d_acc_nodes, d_out_tokens, d_n_new, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_step_out* d_out,

@@ -42,6 +42,7 @@ struct tr_ctx {
   // scratch
   unsigned long long* d_topk_part = nullptr;  // [batch*N][segs][k] packed (value, index) keys
   unsigned int* d_topk_ticket = nullptr;      // [batch*N]
+  unsigned int* d_seq_ticket = nullptr;       // [batch]: CTAs of a sequence that passed tr_commit's read phase
   int topk_segs = 0;
   float* d_attn_part_o = nullptr;   // [slots][128][128]
   float* d_attn_part_ml = nullptr;  // [slots][128][2]
@@ -52,6 +53,8 @@ struct tr_ctx {
 // launchers (host functions defined next to their kernels)
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s);
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s);
+tr_status tr_launch_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,
+                           const int32_t* d_out_tokens, const int32_t* d_n_new, cudaStream_t s);
 tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);
 tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_mma_setup();

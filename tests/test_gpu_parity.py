@@ -291,6 +291,80 @@ def test_attention_other_workload_shapes_one_layer_sampled(harness, name):
     dw.close()
 
 
+# ------------------------------------------------------------------ decoder loop with KV / token commit
+def test_decode_loop_with_commit_grows_the_prefix(tr):
+    """Steps of: attention at the current (device-resident) prefix length -> verify/update/retrieve -> commit of the
+    accepted path.  Cache contents, prefix lengths and emitted tokens must equal the oracle's, bit for bit, and the
+    attention output of the last step must match the oracle's attention over the oracle's cache."""
+    B, L, Hq, Hkv, D, N, V, k_cand = 2, 2, 4, 2, 128, 15, 500, 8
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], vocab=V, ctx=(70, 37), n_layers=L, n_q_heads=Hq, n_kv_heads=Hkv,
+                            head_dim=D, boost=5.0)
+    steps, cap_rows, cap_tok = 12, 70 + N + 12 * 7 + 8, 12 * 7 + 4
+    parent, rank = tr.tr_template_from_branching(w.branching, N)
+    ctx = tr.tr_init(V, k_cand, parent, rank, batch=B)
+    rng = np.random.default_rng(5)
+    bits = lambda shape: synth.f32_to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    k_h, v_h = bits((B, L, Hkv, cap_rows, D)), bits((B, L, Hkv, cap_rows, D))
+    q_h = bits((B, L, N, Hq, D))
+    from paper_2408_08696_b200.harness import bf16_tensor
+    dev = torch.device("cuda", 0)
+    d_k, d_v, d_q = bf16_tensor(k_h, dev), bf16_tensor(v_h, dev), bf16_tensor(q_h, dev)
+    d_o = torch.zeros_like(d_q)
+    d_ctx = torch.tensor(list(w.ctx), dtype=torch.int32, device=dev)
+    d_tokens = torch.zeros(B, cap_tok, dtype=torch.int32, device=dev)
+    d_ntok = torch.zeros(B, dtype=torch.int32, device=dev)
+    attn = tr.make_attn_args(ctx, d_q, d_k, d_v, d_o, d_ctx, cap_rows - N)
+    cargs = tr.make_commit_args(ctx, d_k, d_v, d_ctx, d_tokens, d_ntok)
+    out_struct, out = tr.make_step_out(ctx)
+    # integer loop state on both sides
+    M = synth.seeded_matrix(w)
+    for b in range(B):
+        tr.tr_matrix_import(ctx, b, M[b])
+    Mo = [m.astype(np.int64) for m in M]
+    succ, noise = synth.zipf_successors(w), synth.noise_logits(w, 2)
+    roots = synth.root_tokens(w)
+    d_tree = torch.zeros(B, N, dtype=torch.int32, device=dev)
+    tr.tr_build_tree(ctx, torch.from_numpy(roots).to(dev), d_tree)
+    So = [orc.bfs_tree(Mo[b], parent, rank, int(roots[b])) for b in range(B)]
+    c_o, tok_o = list(w.ctx), [[] for _ in range(B)]
+    for s in range(steps):
+        logits = np.stack([synth.step_logits(noise[s % 2, b], So[b], succ, w.boost) for b in range(B)])
+        tr.tr_tree_attention(ctx, attn)
+        tr.tr_verify_update(ctx, torch.from_numpy(logits).to(dev), d_tree, out_struct)
+        tr.tr_commit(ctx, cargs, out["acc_nodes"], out["out_tokens"], out["n_new"])
+        d_tree.copy_(out["next_tree"])
+        torch.cuda.synchronize()
+        if s == steps - 1:                                    # attention of the last step, at the grown prefix
+            for b in range(B):
+                for l in range(L):
+                    ref = orc.tree_attention(synth.bf16_bits_to_f32(q_h[b, l]),
+                                             synth.bf16_bits_to_f32(k_h[b, l, :, : c_o[b] + N]),
+                                             synth.bf16_bits_to_f32(v_h[b, l, :, : c_o[b] + N]), c_o[b], parent)
+                    got = d_o[b, l].float().cpu().numpy()
+                    for h in range(Hq):
+                        mx, rel = attention_close(got[:, h], ref[:, h])
+                        assert mx <= ATOL and rel <= RTOL, (b, l, h, mx, rel)
+        for b in range(B):
+            rec = orc.verify_update(Mo[b], So[b], logits[b], parent, rank)
+            c_o[b], tok_o[b] = orc.commit(k_h[b], v_h[b], c_o[b], tok_o[b], rec["acc_nodes"], rec["out_tokens"])
+            So[b] = rec["next_tree"]
+        assert d_ctx.cpu().tolist() == c_o
+        assert d_ntok.cpu().tolist() == [len(t) for t in tok_o]
+    assert tr.tr_device_flags(ctx) == 0
+    for b in range(B):
+        assert d_tokens[b, : len(tok_o[b])].cpu().tolist() == tok_o[b]
+        assert len(tok_o[b]) > steps                           # some drafts were accepted along the way
+    assert (d_k.view(torch.int16).cpu().numpy().view(np.uint16) == k_h).all()
+    assert (d_v.view(torch.int16).cpu().numpy().view(np.uint16) == v_h).all()
+    # a cache without room for another tree: flagged, sequence left untouched
+    d_ctx[0] = cap_rows - N
+    before = d_ctx.clone()
+    tr.tr_commit(ctx, cargs, out["acc_nodes"], out["out_tokens"], out["n_new"])
+    assert tr.tr_device_flags(ctx) & tr.TR_FLAG_CACHE_FULL
+    assert d_ctx[0].item() == before[0].item()
+    tr.tr_destroy(ctx)
+
+
 # ------------------------------------------------------------------ whole step, host-buffer entry point
 def test_step_host_matches_device_calls(harness, tr):
     import ctypes as C

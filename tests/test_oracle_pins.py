@@ -368,3 +368,20 @@ def test_synth_is_seeded_and_shaped():
     lg = synth.step_logits(a[0, 0], np.zeros(15, dtype=np.int64), succ, 4.0)
     assert np.count_nonzero(lg != a[0, 0]) == 15
     assert len(synth.WORKLOADS["llama2-70b-b8"].ctx) == 8
+
+
+# ---------------------------------------------------------------- commit of the accepted path
+def test_commit_hand_example_and_gather_property():
+    # tree rows sit at 3..8 of a 10-row cache (prefix C = 3, N = 6); accepted path = nodes 0, 2, 5
+    k = np.arange(10, dtype=np.float64)[None, :, None] * np.ones((2, 1, 4)) + np.array([0.0, 100.0])[:, None, None]
+    v = -k.copy()
+    k0, v0 = k.copy(), v.copy()
+    c, toks = orc.commit(k, v, 3, [9, 9, 9], [0, 2, 5], [41, 42, 43])
+    assert c == 6 and toks == [9, 9, 9, 41, 42, 43]
+    assert k[0, :, 0].tolist() == [0, 1, 2, 3, 5, 8, 6, 7, 8, 9]          # rows 3,4,5 <- old rows 3,5,8
+    assert (k[:, 3:6] == k0[:, [3, 5, 8]]).all() and (v[:, 3:6] == v0[:, [3, 5, 8]]).all()
+    assert (k[:, :3] == k0[:, :3]).all() and (k[:, 6:] == k0[:, 6:]).all()  # nothing else moves
+    # overlapping case: a later destination is an earlier source (path 0, 1, 2 after 0, 2, ... is impossible; use 0,2,3)
+    k = k0.copy(); v = v0.copy()
+    orc.commit(k, v, 3, [], [0, 2, 3], [1, 2, 3])
+    assert k[0, 3:6, 0].tolist() == [3, 5, 6]
