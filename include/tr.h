@@ -145,7 +145,22 @@ typedef struct {
 } tr_step_out;
 tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const int32_t* d_tree, const tr_step_out* out,
                            void* stream);
-int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appendix: maximum acceptance length) */
+int32_t tr_max_new_tokens(const tr_ctx* ctx);
+
+/*
+ * Update-rule variants the paper compares (Sec. 5.2 "Update Strategies" and "Effect of Rejected Tokens"; Appendix
+ * "Explanation of Three Update Strategies").  Takes effect for the following tr_verify_update calls.
+ *   rule : TR_UPDATE_LAST  (default) - a repeated token keeps the row of its last occurrence
+ *          TR_UPDATE_FIRST           - ... of its first occurrence
+ *   scope: TR_UPDATE_ALL_DRAFT (default) - every node of the tree updates its token's row
+ *          TR_UPDATE_ONLY_ACCEPTED       - only the nodes of the accepted path do
+ * The paper's own uncontrolled update ("Cur") is a data race by design and is not offered.
+ */
+#define TR_UPDATE_LAST 0
+#define TR_UPDATE_FIRST 1
+#define TR_UPDATE_ALL_DRAFT 0
+#define TR_UPDATE_ONLY_ACCEPTED 1
+tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope); /* depth of the template + 1 (Appendix: maximum acceptance length) */
 
 /*
  * Commit the accepted path (Sec. 5.4: a step ends by "updating the matrix, input tokens, and key-value cache").

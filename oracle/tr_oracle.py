@@ -191,16 +191,26 @@ def accept(S, argmax, parent):
 # --------------------------------------------------------------------------
 # Matrix update (Sec. 3.3; Appendix "Explanation of Three Update Strategies")
 # --------------------------------------------------------------------------
-def update_matrix(M, S, O):
+def update_matrix(M, S, O, rule="last", nodes=None):
     """M[S[i]] <- O[i] for every node of the merged sequence, root and rejected
     nodes included, applied in increasing i: a token that occurs several times
     keeps the row of its last occurrence (the appendix's "Last" strategy, which
     is one of the outcomes the uncontrolled parallel update may produce).
+    rule="first" is the appendix's "First" strategy (positions of each token's
+    first occurrence); `nodes` restricts the update to a subset of the nodes
+    (the "only accepted" setting of Sec. 5.2, Table 4).
     In place; also returns M.
-    Pinned by: the appendix's worked example S = [a, b, c, a, d].
+    Pinned by: the appendix's worked example S = [a, b, c, a, d] for both rules.
     """
-    for i in range(len(S)):
-        M[S[i], :] = O[i, :]
+    idx = list(range(len(S))) if nodes is None else sorted(int(i) for i in nodes)
+    if rule == "last":
+        for i in idx:
+            M[S[i], :] = O[i, :]
+    elif rule == "first":
+        for i in reversed(idx):      # going backwards, the first occurrence is written last
+            M[S[i], :] = O[i, :]
+    else:
+        raise ValueError(rule)
     return M
 
 
@@ -244,7 +254,7 @@ def bfs_tree(M, parent, rank, root):
 # --------------------------------------------------------------------------
 # One whole step
 # --------------------------------------------------------------------------
-def verify_update(M, S, logits, parent, rank):
+def verify_update(M, S, logits, parent, rank, rule="last", only_accepted=False):
     """argtopk -> accept -> update M -> next tree from the updated M, rooted at
     the last confirmed token (the retrieve / verify / update cycle of Sec. 3 and
     Sec. 5.4).  M is modified in place.
@@ -253,7 +263,7 @@ def verify_update(M, S, logits, parent, rank):
     k = M.shape[1]
     O = argtopk(logits, k)
     n_new, acc_nodes, out_tokens, next_root = accept(S, O[:, 0], parent)
-    update_matrix(M, S, O)
+    update_matrix(M, S, O, rule=rule, nodes=acc_nodes if only_accepted else None)
     nxt = bfs_tree(M, parent, rank, next_root)
     return dict(topk=O, n_new=n_new, acc_nodes=acc_nodes, out_tokens=out_tokens,
                 next_root=next_root, next_tree=nxt)

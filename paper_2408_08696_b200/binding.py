@@ -28,6 +28,7 @@ TR_OK = 0
 TR_ERR_INVALID_ARG, TR_ERR_TEMPLATE, TR_ERR_UNSUPPORTED, TR_ERR_CUDA, TR_ERR_NOMEM, TR_ERR_DEVICE_FLAG = -1, -2, -3, -4, -5, -6
 TR_FLAG_BAD_TOKEN, TR_FLAG_WAIT_TIMEOUT, TR_FLAG_CACHE_FULL = 1, 2, 4
 TR_MAX_NODES, TR_MAX_K = 128, 16
+TR_UPDATE_LAST, TR_UPDATE_FIRST, TR_UPDATE_ALL_DRAFT, TR_UPDATE_ONLY_ACCEPTED = 0, 1, 0, 1
 
 
 class TrError(RuntimeError):
@@ -83,6 +84,7 @@ lib.tr_build_tree.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.tr_tree_attention.argtypes = [C.c_void_p, C.POINTER(tr_attn_args), C.c_void_p]
 lib.tr_verify_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(tr_step_out), C.c_void_p]
 lib.tr_max_new_tokens.argtypes = [C.c_void_p]
+lib.tr_set_update_rule.argtypes = [C.c_void_p, C.c_int32, C.c_int32]
 lib.tr_device_flags.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
 lib.tr_step_host.argtypes = [C.c_void_p, C.POINTER(tr_attn_args), C.POINTER(tr_step_out), C.POINTER(tr_host_io),
                              C.c_void_p]
@@ -264,6 +266,10 @@ def tr_commit(ctx, args, d_acc_nodes, d_out_tokens, d_n_new, stream=None):
     _check(lib.tr_commit(ctx.handle, C.byref(args), _dev(d_acc_nodes, torch.int32, "d_acc_nodes"),
                          _dev(d_out_tokens, torch.int32, "d_out_tokens"), _dev(d_n_new, torch.int32, "d_n_new"),
                          _stream(stream)), "tr_commit")
+
+
+def tr_set_update_rule(ctx, rule=TR_UPDATE_LAST, scope=TR_UPDATE_ALL_DRAFT):
+    _check(lib.tr_set_update_rule(ctx.handle, rule, scope), "tr_set_update_rule")
 
 
 def tr_device_flags(ctx):

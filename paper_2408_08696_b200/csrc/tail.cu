@@ -73,7 +73,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
                const int32_t* __restrict__ level_off, int depth_max, const int32_t* tree_in,
                const int32_t* __restrict__ topk_idx, int32_t* __restrict__ n_new, int32_t* __restrict__ acc_nodes,
                int32_t* __restrict__ out_tokens, int32_t* __restrict__ next_root, int32_t* tree_out,
-               uint32_t* __restrict__ flags) {
+               uint32_t* __restrict__ flags, const uint32_t* __restrict__ anc, int update_rule, int update_scope) {
   __shared__ int32_t s_S[TR_MAX_NODES];
   __shared__ int32_t s_argmax[TR_MAX_NODES];
   __shared__ int32_t s_tree[TR_MAX_NODES];
@@ -138,10 +138,23 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     s_tree[0] = bonus;
   }
 
-  // ---- update: last occurrence of each token writes its whole row
-  if (tid < n && tok_ok) {
+  // ---- update: one occurrence of each token writes its whole row - the last one by default, the first one
+  //      under TR_UPDATE_FIRST; under TR_UPDATE_ONLY_ACCEPTED only nodes on the accepted path take part
+  //      (node i is on it iff i is the accepted leaf or one of its ancestors: bit i of the leaf's mask)
+  uint32_t in_scope = 1u;
+  if (update_scope == TR_UPDATE_ONLY_ACCEPTED && tid < n) in_scope = (anc[leaf * 4 + (tid >> 5)] >> (tid & 31)) & 1u;
+  if (update_scope == TR_UPDATE_ONLY_ACCEPTED) {  // the competitors below must be in scope too
+    __syncthreads();                               // (everyone is past reading s_S for the acceptance walk)
+    if (tid < n && !in_scope) s_S[tid] = -1 - tid;  // a value no token equals
+    __syncthreads();
+  }
+  if (tid < n && tok_ok && in_scope) {
     bool last = true;
-    for (int j = tid + 1; j < n; ++j) last = last && (s_S[j] != tok);
+    if (update_rule == TR_UPDATE_FIRST) {
+      for (int j = 0; j < tid; ++j) last = last && (s_S[j] != tok);
+    } else {
+      for (int j = tid + 1; j < n; ++j) last = last && (s_S[j] != tok);
+    }
     if (last) {
       int32_t* dst = M + static_cast<size_t>(tok) * k;
 #pragma unroll
@@ -167,7 +180,7 @@ tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* 
                                                      ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
                                                      d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes,
                                                      out->d_out_tokens, out->d_next_root, out->d_next_tree,
-                                                     ctx->d_flags);
+                                                     ctx->d_flags, ctx->d_anc, ctx->update_rule, ctx->update_scope);
   TR_CUDA_TRY(cudaGetLastError());
   return TR_OK;
 }

@@ -169,6 +169,15 @@ extern "C" tr_status tr_destroy(tr_ctx* ctx) {
   return free_all(ctx);
 }
 
+extern "C" tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope) {
+  if (!ctx || (rule != TR_UPDATE_LAST && rule != TR_UPDATE_FIRST) ||
+      (scope != TR_UPDATE_ALL_DRAFT && scope != TR_UPDATE_ONLY_ACCEPTED))
+    return TR_ERR_INVALID_ARG;
+  ctx->update_rule = rule;
+  ctx->update_scope = scope;
+  return TR_OK;
+}
+
 extern "C" int32_t tr_max_new_tokens(const tr_ctx* ctx) { return ctx ? ctx->depth_max + 1 : 0; }
 
 extern "C" tr_status tr_matrix_zero(tr_ctx* ctx, void* stream) {

@@ -47,6 +47,7 @@ struct tr_ctx {
   float* d_attn_part_o = nullptr;   // [slots][128][128]
   float* d_attn_part_ml = nullptr;  // [slots][128][2]
   uint32_t* d_flags = nullptr;
+  int update_rule = 0, update_scope = 0;  // TR_UPDATE_*
   bool force_mma = false;  // debugging aid: TR_ATTN_FORCE_MMA=1 at tr_init keeps head_dim 128 on the warp-MMA kernel
 };
 

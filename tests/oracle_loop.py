@@ -7,8 +7,9 @@ from paper_2408_08696_b200 import synth
 
 
 class OracleLoop:
-    def __init__(self, w, n_rot=4, zero_matrix=False):
+    def __init__(self, w, n_rot=4, zero_matrix=False, rule="last", only_accepted=False):
         self.w = w
+        self.rule, self.only_accepted = rule, only_accepted
         self.parent, self.rank = orc.template_from_branching(w.branching, w.n_nodes)
         self.M = [np.zeros((w.vocab, w.k), dtype=np.int64) if zero_matrix else m.astype(np.int64)
                   for m in synth.seeded_matrix(w)]
@@ -23,7 +24,8 @@ class OracleLoop:
         recs = []
         for b in range(self.w.batch):
             logits = synth.step_logits(self.noise[r, b], self.S[b], self.succ, self.w.boost)
-            rec = orc.verify_update(self.M[b], self.S[b], logits, self.parent, self.rank)
+            rec = orc.verify_update(self.M[b], self.S[b], logits, self.parent, self.rank, rule=self.rule,
+                                    only_accepted=self.only_accepted)
             self.S[b] = rec["next_tree"]
             recs.append(rec)
         return recs

@@ -168,6 +168,25 @@ def test_loop_large_vocab(harness):
     _run_loop(harness, synth.WORKLOADS["llama3-8b"], 6)
 
 
+@pytest.mark.parametrize("rule,only_accepted", [("first", False), ("last", True), ("first", True)])
+@pytest.mark.parametrize("zero_matrix", [False, True])
+def test_loop_update_rule_variants(harness, tr, rule, only_accepted, zero_matrix):
+    """The update strategies the paper compares (First / Last, all drafts / only accepted); the zero matrix makes
+    every draft the same token, so the duplicate handling decides every row."""
+    w = synth.WORKLOADS["tiny"]
+    dw = harness.DeviceWorkload(w, with_attention=False, zero_matrix=zero_matrix)
+    tr.tr_set_update_rule(dw.ctx, tr.TR_UPDATE_FIRST if rule == "first" else tr.TR_UPDATE_LAST,
+                          tr.TR_UPDATE_ONLY_ACCEPTED if only_accepted else tr.TR_UPDATE_ALL_DRAFT)
+    ol = OracleLoop(w, zero_matrix=zero_matrix, rule=rule, only_accepted=only_accepted)
+    for i in range(25):
+        dw.step(i)
+        compare_step(ol.step(i), dw.snapshot(), dw.ctx.max_new)
+    assert (tr.tr_matrix_export(dw.ctx, 0) == ol.M[0]).all()
+    with pytest.raises(tr.TrError):
+        tr.tr_set_update_rule(dw.ctx, 7, 0)
+    dw.close()
+
+
 def test_duplicate_tokens_last_writer_wins(tr):
     # Appendix "Explanation of Three Update Strategies": S = [a, b, c, a, d] keeps O[3] for a.
     parent = np.array([-1, 0, 0, 0, 0], dtype=np.int32)
@@ -234,6 +253,17 @@ def test_attention_gqa_and_batch_with_mixed_contexts(harness):
     w = dataclasses.replace(synth.WORKLOADS["llama2-70b-b8"], n_q_heads=8, n_kv_heads=2, ctx=(100, 257, 31))
     _attention_case(harness, w, 2)
     _attention_case(harness, w, 1, splits=3)
+
+
+def test_largest_tree_128_nodes_attention_and_loop(harness):
+    # the maximum template size (ancestor masks are 128-bit; the attention tile has 128 query rows)
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], branching=(10, 10), n_nodes=128, n_q_heads=2, n_kv_heads=2,
+                            ctx=(200,), vocab=3000, k=16)
+    _attention_case(harness, w, 1)
+    _attention_case(harness, w, 1, splits=3)
+    w64 = dataclasses.replace(w, head_dim=64)
+    _attention_case(harness, w64, 1)
+    _run_loop(harness, w, 6)
 
 
 def test_attention_single_node_tree(harness):

@@ -308,6 +308,14 @@ def test_update_last_writer_matches_appendix_example(golden_dir):
     assert M[11].tolist() == g["M[b]"] and M[12].tolist() == g["M[c]"] and M[13].tolist() == g["M[d]"]
     untouched = [i for i in range(20) if i not in (10, 11, 12, 13)]
     assert (M[untouched] == -1).all()
+    # "First": positions of each token's first occurrence
+    M1 = np.full((20, 4), -1, dtype=np.int64)
+    orc.update_matrix(M1, S, O, rule="first")
+    assert M1[10].tolist() == g["M[a] first"] and M1[13].tolist() == g["M[d]"] and (M1[untouched] == -1).all()
+    # only a subset of the nodes (the "only accepted" setting): others keep their old rows
+    M2 = np.full((20, 4), -1, dtype=np.int64)
+    orc.update_matrix(M2, S, O, nodes=[0, 2])
+    assert M2[10].tolist() == g["M[a] first"] and M2[12].tolist() == g["M[c]"] and (M2[[11, 13]] == -1).all()
 
 
 def test_update_covers_root_and_rejected_nodes():
