@@ -264,6 +264,31 @@ struct TileCursor {
   }
 };
 
+// sm_100 packed / three-input float instructions: half the instruction count of the softmax's element-wise passes
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -496,7 +521,8 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
         for (int q = 0; q < 4; ++q)
 #pragma unroll
-          for (int c = 0; c < 32; ++c) mx[c & 7] = fmaxf(mx[c & 7], __uint_as_float(sreg[q][c]));
+          for (int c = 0; c < 32; c += 2)  // three-input max: two scores per instruction
+            mx[(c >> 1) & 7] = max3(mx[(c >> 1) & 7], __uint_as_float(sreg[q][c]), __uint_as_float(sreg[q][c + 1]));
         const float tmax = fmaxf(fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3])),
                                  fmaxf(fmaxf(mx[4], mx[5]), fmaxf(mx[6], mx[7]))) * p.scale_log2;
         // lazy rescale: keep the old reference unless the maximum grew by more than 2^8
@@ -525,20 +551,23 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         }
         l *= alpha;
         const float nsub = (m_ref == -INFINITY) ? 0.f : -m_ref;
-        float sm4[4] = {0.f, 0.f, 0.f, 0.f};
+        const uint64_t scale2 = pack2(p.scale_log2, p.scale_log2), nsub2 = pack2(nsub, nsub);
+        uint64_t sm2[4] = {0ull, 0ull, 0ull, 0ull};  // packed (even, odd) partial row sums
         uint32_t preg[2][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q)
 #pragma unroll
           for (int c = 0; c < 32; c += 2) {
-            const float p0 = fast_exp2(fmaf(__uint_as_float(sreg[q][c]), p.scale_log2, nsub));
-            const float p1 = fast_exp2(fmaf(__uint_as_float(sreg[q][c + 1]), p.scale_log2, nsub));
-            sm4[(c >> 1) & 1] += p0;
-            sm4[2 + ((c >> 1) & 1)] += p1;
+            float x0, x1;
+            unpack2(fma2(pack2(__uint_as_float(sreg[q][c]), __uint_as_float(sreg[q][c + 1])), scale2, nsub2), x0, x1);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            sm2[(c >> 1) & 3] = add2(sm2[(c >> 1) & 3], pack2(p0, p1));
             __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
             preg[q >> 1][(q & 1) * 16 + (c >> 1)] = *reinterpret_cast<uint32_t*>(&pk);
           }
-        const float sum = (sm4[0] + sm4[1]) + (sm4[2] + sm4[3]);
+        float se, so;
+        unpack2(add2(add2(sm2[0], sm2[1]), add2(sm2[2], sm2[3])), se, so);
+        const float sum = se + so;
         l += sum;
         tc_st32(tmem + lane_base + sb * 128u, preg[0]);
         tc_st32(tmem + lane_base + sb * 128u + 32u, preg[1]);
