@@ -181,13 +181,15 @@ def run_ours(args, w):
     graphs = dw.capture_graphs()
     if args.profile:
         for i in range(W + K):
-            graphs[i % dw.n_rot].replay()
+            graphs[i % dw.n_rot].replay()  # rotation order
         torch.cuda.synchronize()
         dw.close()
         return
     stream = torch.cuda.current_stream()
-    for i in range(W):
-        graphs[i % dw.n_rot].replay()
+    step_no = 0  # the graphs must be replayed in rotation order (each patches the next one's logits)
+    for _ in range(W):
+        graphs[step_no % dw.n_rot].replay()
+        step_no += 1
     torch.cuda.synchronize()
 
     # ---- timed region: K graph replays back to back, device time between two events on the launching stream
@@ -196,8 +198,9 @@ def run_ours(args, w):
     sampler = ClockSampler(local_rank) if rank == 0 else None
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for i in range(K):
-        graphs[(W + i) % dw.n_rot].replay()
+    for _ in range(K):
+        graphs[step_no % dw.n_rot].replay()
+        step_no += 1
     e1.record(stream)
     torch.cuda.synchronize()
     replicas.barrier()
@@ -206,19 +209,19 @@ def run_ours(args, w):
         # the timed region lasts tens of milliseconds; keep the same load running (untimed) for about half a second
         # so that nvidia-smi's 100 ms samples see the clocks under this load
         t_end = time.perf_counter() + 0.6
-        i = 0
         while time.perf_counter() < t_end:
             for _ in range(50):
-                graphs[(W + K + i) % dw.n_rot].replay()
-                i += 1
+                graphs[step_no % dw.n_rot].replay()
+                step_no += 1
             torch.cuda.synchronize()
     clocks = sampler.stop() if sampler else None
     agg = replicas.aggregate(elapsed_ms, K, device=dev if world > 1 else "cpu")
     flags = tr.tr_device_flags(dw.ctx)
     # acceptance statistic of the toy model (a sanity figure, not a result): 64 untimed steps, n_new read each step
     n_new_sum, n_stat = 0, 64
-    for i in range(n_stat):
-        graphs[i % dw.n_rot].replay()
+    for _ in range(n_stat):
+        graphs[step_no % dw.n_rot].replay()
+        step_no += 1
         n_new_sum += int(dw.out["n_new"].sum().item())
 
     # ---- dominant kernel (tree attention) alone: event pair around every launch, same stream

@@ -88,8 +88,11 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   int32_t tok = 0;
   int32_t row[TR_MAX_K];
   bool tok_ok = false;
+  if (tid < n) tok = tree_in[static_cast<size_t>(b) * n + tid];  // written by an earlier step, not by the top-k kernel
+  // Everything above was fetched while the top-k kernel may still have been running (programmatic dependent
+  // launch); its output is read only from here on.
+  tr_grid_dependency_wait();
   if (tid < n) {
-    tok = tree_in[static_cast<size_t>(b) * n + tid];
     tok_ok = (tok >= 0 && tok < V);
     if (!tok_ok) atomicOr(flags, TR_FLAG_BAD_TOKEN);
     s_S[tid] = tok;
@@ -176,11 +179,10 @@ tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tr
 }
 
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s) {
-  tr_tail_kernel<<<ctx->batch, TAIL_THREADS, 0, s>>>(ctx->d_M, ctx->vocab, ctx->k, ctx->n_nodes, ctx->d_parent,
-                                                     ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
-                                                     d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes,
-                                                     out->d_out_tokens, out->d_next_root, out->d_next_tree,
-                                                     ctx->d_flags, ctx->d_anc, ctx->update_rule, ctx->update_scope);
-  TR_CUDA_TRY(cudaGetLastError());
+  TR_CUDA_TRY(tr_launch_pdl(tr_tail_kernel, dim3(ctx->batch), dim3(TAIL_THREADS), 0, s, ctx->d_M, ctx->vocab, ctx->k,
+                            ctx->n_nodes, ctx->d_parent, ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
+                            d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes, out->d_out_tokens,
+                            out->d_next_root, out->d_next_tree, ctx->d_flags, ctx->d_anc, ctx->update_rule,
+                            ctx->update_scope));
   return TR_OK;
 }

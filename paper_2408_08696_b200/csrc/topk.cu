@@ -48,6 +48,8 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const float* rowp = logits + static_cast<size_t>(row) * V;
   const int seg_base = seg * TOPK_SEG_ELEMS;
+  // (programmatic dependent launch) the logits belong to whatever ran before on this stream
+  tr_grid_dependency_wait();
 
   // ---- (1) 16 values per thread in registers; running maximum with its index (first = lowest index wins ties)
   float v[E];
@@ -212,12 +214,11 @@ tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx
   dim3 grid(ctx->topk_segs, rows);
   const bool vec = (ctx->vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
   if (vec)
-    tr_topk_kernel<true><<<grid, TOPK_THREADS, 0, s>>>(d_logits, ctx->vocab, ctx->k, ctx->topk_segs,
-                                                       ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx);
+    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, ctx->k,
+                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx));
   else
-    tr_topk_kernel<false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, ctx->vocab, ctx->k, ctx->topk_segs,
-                                                        ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx);
-  TR_CUDA_TRY(cudaGetLastError());
+    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, ctx->k,
+                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx));
   return TR_OK;
 }
 

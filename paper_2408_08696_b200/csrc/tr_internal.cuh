@@ -51,6 +51,27 @@ struct tr_ctx {
   bool force_mma = false;  // debugging aid: TR_ATTN_FORCE_MMA=1 at tr_init keeps head_dim 128 on the warp-MMA kernel
 };
 
+// Launch with programmatic dependent launch: the kernel may be scheduled while the previous kernel of the stream is
+// still draining; it must execute tr_grid_dependency_wait() before it touches anything that kernel wrote.
+template <typename... KArgs, typename... Args>
+inline cudaError_t tr_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                 Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#ifdef __CUDACC__
+__device__ __forceinline__ void tr_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // launchers (host functions defined next to their kernels)
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s);
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s);

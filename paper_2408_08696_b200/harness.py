@@ -52,34 +52,36 @@ class DeviceWorkload:
                                           splits=splits)
         torch.cuda.synchronize(self.dev)
 
-    # one whole step: toy-model logits for the current tree, attention over all layers, verify/update/retrieve
-    def step(self, i, stream=None, side=None):
-        """`side`: optional second stream for the toy model's logits patch.  The patch is harness work (a real
-        model's logits come out of its LM head), so the graphs run it beside the attention launch instead of in
-        front of it; the step's own kernels stay in order on `stream`."""
-        r = i % self.n_rot
-        main = torch.cuda.current_stream(self.dev) if stream is None else stream
-        patch_stream = main if side is None else side
-        if side is not None:
-            side.wait_stream(main)
+    def patch(self, r, stream=None):
+        """Toy model: rewrite the tree-dependent entries of rotating logits buffer r for the current tree."""
         tr.trs_patch_logits(self.d_logits[r], self.d_noise[r], self.d_tree, self.d_prev_col[r], self.d_succ,
-                            self.w.boost, patch_stream)
+                            self.w.boost, stream)
+
+    # one whole step: toy-model logits for the current tree, attention over all layers, verify/update/retrieve
+    def step(self, i, stream=None):
+        r = i % self.n_rot
+        self.patch(r, stream)
         if self.attn is not None:
-            tr.tr_tree_attention(self.ctx, self.attn, main)
-        if side is not None:
-            main.wait_stream(side)
-        tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, main)
+            tr.tr_tree_attention(self.ctx, self.attn, stream)
+        tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, stream)
 
     def capture_graphs(self):
-        """One CUDA graph per rotating logits buffer; replay graphs[i % n_rot] for step i."""
+        """One CUDA graph per rotating logits buffer; replay graphs[i % n_rot] for step i = 0, 1, 2, ... in order.
+        Graph r holds the step's own kernels - attention, top-k, accept/update/retrieve - followed by the toy
+        model's patch of buffer r+1 for the NEXT step (the harness work sits at the end of the chain instead of
+        in front of the attention launch); buffer 0 is patched here, eagerly, for the first replay."""
         graphs = []
         s = torch.cuda.Stream(self.dev)
-        side = torch.cuda.Stream(self.dev)
+        self.patch(0)
+        torch.cuda.synchronize(self.dev)
         with torch.cuda.stream(s):
             for r in range(self.n_rot):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=s):
-                    self.step(r, stream=s, side=side if self.attn is not None else None)
+                    if self.attn is not None:
+                        tr.tr_tree_attention(self.ctx, self.attn, s)
+                    tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, s)
+                    self.patch((r + 1) % self.n_rot, s)
                 graphs.append(g)
         torch.cuda.synchronize(self.dev)
         return graphs
