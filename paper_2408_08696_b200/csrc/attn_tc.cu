@@ -58,8 +58,12 @@ struct TcParams {
   float* part_o;
   float* part_ml;
   uint32_t* flags;
-  int N, Hq, Hkv, L, S, n_units;
-  uint32_t div_group[2], div_S[2], div_Hkv[2], div_L[2];  // (multiplier, shift) for exact u32 division
+  int N, L, S, n_units;
+  // Query rows are grouped per "head unit" hu: with grouped-query attention the G query heads that share a KV head
+  // are packed into common 128-row tiles (row = node * G + head-in-group), MT tiles per head unit; when the group
+  // size does not divide 128, every query head is its own head unit (G = 1) and kv_div maps it to its KV head.
+  int HU, G, g_shift, MT, kv_div;
+  uint32_t div_MT[2], div_S[2], div_HU[2], div_L[2], div_kv[2];  // (multiplier, shift) for exact u32 division
   int64_t os_b, os_h, os_t, os_l;
   float scale_log2;
 };
@@ -206,7 +210,7 @@ __host__ __device__ constexpr uint32_t make_idesc(bool b_mn_major) {
 }
 
 struct Unit {
-  int b, layer, kvh, h, split, slot;
+  int b, layer, kvh, h0, node0, split, slot;  // h0: first query head of the tile's rows; node0: its first tree node
   int t0, t1, C;
 };
 
@@ -220,14 +224,15 @@ constexpr int CTX_CACHE = 64;  // context lengths of the first 64 sequences are 
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, int u, const int* s_ctx) {
   Unit x;
   x.slot = u;
-  const uint32_t group = static_cast<uint32_t>(p.Hq / p.Hkv);  // (one divide, by values fixed for the launch)
   uint32_t v = static_cast<uint32_t>(u), q;
-  q = fast_div(v, p.div_group); const uint32_t gq = v - q * group; v = q;
+  q = fast_div(v, p.div_MT); const uint32_t mt = v - q * p.MT; v = q;
   q = fast_div(v, p.div_S); x.split = static_cast<int>(v - q * p.S); v = q;
-  q = fast_div(v, p.div_Hkv); x.kvh = static_cast<int>(v - q * p.Hkv); v = q;
+  q = fast_div(v, p.div_HU); const uint32_t hu = v - q * p.HU; v = q;
   q = fast_div(v, p.div_L); x.layer = static_cast<int>(v - q * p.L); v = q;
   x.b = static_cast<int>(v);
-  x.h = x.kvh * static_cast<int>(group) + static_cast<int>(gq);
+  x.h0 = static_cast<int>(hu) * p.G;
+  x.node0 = static_cast<int>(mt) * (128 >> p.g_shift);
+  x.kvh = static_cast<int>(fast_div(hu, p.div_kv));
   x.C = x.b < CTX_CACHE ? s_ctx[x.b] : p.ctx_len[x.b];
   const int T = (x.C + p.N + BK - 1) / BK;
   x.t0 = static_cast<int>(static_cast<int64_t>(T) * x.split / p.S);
@@ -313,7 +318,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int* s_ctx = reinterpret_cast<int*>(base_ptr + SM_CTX);
   {
-    const int nb = p.n_units / (p.L * p.Hq * p.S);  // sequences
+    const int nb = p.n_units / (p.L * p.HU * p.S * p.MT);  // sequences
     if (tid >= 64 && tid - 64 < CTX_CACHE && tid - 64 < nb) s_ctx[tid - 64] = p.ctx_len[tid - 64];
   }
 
@@ -361,8 +366,9 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ok = mbar_wait(bar(BAR_QEMPTY + qb), ((ui >> 1) & 1u) ^ 1u, s_abort);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_QFULL + qb), TILE_BYTES);
-        tma_load_5d(base + SM_Q + qb * TILE_BYTES, &map_q, bar(BAR_QFULL + qb), 0, x.h, 0, x.layer, x.b);
-        tma_load_5d(base + SM_Q + qb * TILE_BYTES + HALF_BYTES, &map_q, bar(BAR_QFULL + qb), 64, x.h, 0, x.layer, x.b);
+        tma_load_5d(base + SM_Q + qb * TILE_BYTES, &map_q, bar(BAR_QFULL + qb), 0, x.h0, x.node0, x.layer, x.b);
+        tma_load_5d(base + SM_Q + qb * TILE_BYTES + HALF_BYTES, &map_q, bar(BAR_QFULL + qb), 64, x.h0, x.node0, x.layer,
+                    x.b);
         for (int t = x.t0; t < x.t1 && ok; ++t) {
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
@@ -459,13 +465,16 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int r = (warp & 3) * 32 + lane;                 // query row == TMEM lane
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     uint32_t anc[4];
-#pragma unroll
-    for (int w = 0; w < 4; ++w) anc[w] = r < p.N ? p.anc[r * 4 + w] : 0u;
     uint32_t ui = 0, g = 0;
     bool ok = true;
     for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
       const Unit x = decode_unit(p, u, s_ctx);
       const int nt = x.t1 - x.t0;
+      {  // this row's tree node (rows of a packed tile are node-major) and its ancestor mask
+        const int node = x.node0 + (r >> p.g_shift);
+#pragma unroll
+        for (int w = 0; w < 4; ++w) anc[w] = (nt > 0 && node < p.N) ? p.anc[node * 4 + w] : 0u;
+      }
       float m_ref = -INFINITY, l = 0.f;
       const uint32_t ob = ui & 1u;
       for (int j = 0; j < nt && ok; ++j, ++g) {
@@ -603,10 +612,13 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
       const Unit x = decode_unit(p, u, s_ctx);
       const int nt = x.t1 - x.t0;
+      const int node = x.node0 + (r >> p.g_shift);      // rows of a packed tile are node-major ...
+      const int head = x.h0 + (r & (p.G - 1));          // ... with the group's query heads interleaved
+      const bool row_ok = node < p.N;
       float* po = p.part_o + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 128;
       float* pml = p.part_ml + (static_cast<size_t>(x.slot) * ATTN_PART_ROWS + r) * 2;
       if (nt <= 0) {  // empty split: contributes nothing
-        if (p.S > 1 && r < p.N) {
+        if (p.S > 1 && row_ok) {
           pml[0] = -INFINITY;
           pml[1] = 0.f;
         }
@@ -620,7 +632,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       if (tid == 0) USTAMP(3, ui, 0)
       const float l = s_lm[ob * 256 + r], m_ref = s_lm[ob * 256 + 128 + r];
       const float inv = 1.f / l;
-      __nv_bfloat16* orow = p.out + x.b * p.os_b + x.layer * p.os_l + x.h * p.os_h + static_cast<int64_t>(r) * p.os_t;
+      __nv_bfloat16* orow = p.out + x.b * p.os_b + x.layer * p.os_l + head * p.os_h + static_cast<int64_t>(node) * p.os_t;
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         uint32_t oreg[32];
@@ -630,7 +642,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           tc_fence_before();
           mbar_arrive(bar(BAR_OFREE + ob));
         }
-        if (r < p.N) {
+        if (row_ok) {
           if (p.S == 1) {
 #pragma unroll
             for (int c = 0; c < 32; c += 8) {
@@ -652,7 +664,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
           }
         }
       }
-      if (p.S > 1 && r < p.N) {
+      if (p.S > 1 && row_ok) {
         pml[0] = m_ref;
         pml[1] = l;
       }
@@ -707,6 +719,43 @@ bool encode_map(CUtensorMap* m, const void* ptr, const uint64_t (&dims)[5], cons
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Merge of the per-split partials written by tr_attn_tc_kernel: out = sum_s 2^(m_s - m*) O_s / sum_s 2^(m_s - m*) l_s.
+// One CTA per (8 tile rows, tile); 32 lanes x float4 cover the 128 dims of a row.  Slots are numbered like the
+// units: (((b, layer, head unit), split), tile).
+__global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams p) {
+  const int r = blockIdx.x * 8 + (threadIdx.x >> 5);  // row of the tile
+  const int d = (threadIdx.x & 31) * 4;
+  const uint32_t t = blockIdx.y;                        // (b, layer, head unit, tile)
+  const uint32_t blh = t / p.MT, mt = t - blh * p.MT;
+  const uint32_t bl = blh / p.HU, hu = blh - bl * p.HU;
+  const uint32_t b = bl / p.L, layer = bl - b * p.L;
+  const int node = static_cast<int>(mt) * (128 >> p.g_shift) + (r >> p.g_shift);
+  const int head = static_cast<int>(hu) * p.G + (r & (p.G - 1));
+  if (node >= p.N) return;
+  float mstar = -INFINITY;
+  for (int s = 0; s < p.S; ++s) {
+    const size_t slot = (static_cast<size_t>(blh) * p.S + s) * p.MT + mt;
+    mstar = fmaxf(mstar, p.part_ml[(slot * ATTN_PART_ROWS + r) * 2]);
+  }
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float den = 0.f;
+  for (int s = 0; s < p.S; ++s) {
+    const size_t slot = (static_cast<size_t>(blh) * p.S + s) * p.MT + mt;
+    const float2 ml = *reinterpret_cast<const float2*>(p.part_ml + (slot * ATTN_PART_ROWS + r) * 2);
+    const float w = (ml.x == -INFINITY) ? 0.f : exp2f(ml.x - mstar);
+    const float4 o = *reinterpret_cast<const float4*>(p.part_o + (slot * ATTN_PART_ROWS + r) * 128 + d);
+    acc.x += w * o.x; acc.y += w * o.y; acc.z += w * o.z; acc.w += w * o.w;
+    den += w * ml.y;
+  }
+  const float inv = 1.f / den;
+  __nv_bfloat16* op = p.out + b * p.os_b + layer * p.os_l + head * p.os_h + static_cast<int64_t>(node) * p.os_t + d;
+  __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv), hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+  uint2 w2;
+  w2.x = *reinterpret_cast<uint32_t*>(&lo);
+  w2.y = *reinterpret_cast<uint32_t*>(&hi);
+  *reinterpret_cast<uint2*>(op) = w2;
+}
+
 }  // namespace
 
 tr_status tr_attention_tc_setup() {
@@ -714,7 +763,6 @@ tr_status tr_attention_tc_setup() {
   return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
 }
 
-void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
 
 // (M, k) with floor(u / d) == (u * M) >> k for all 0 <= u < 2^31: k = 31 + ceil(log2 d), M = ceil(2^k / d) < 2^32.
 static void magic_u32(uint32_t d, uint32_t (&ms)[2]) {
@@ -727,32 +775,42 @@ static void magic_u32(uint32_t d, uint32_t (&ms)[2]) {
 
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s) {
   if (a->head_dim != HD) return TR_ERR_UNSUPPORTED;
-  const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * a->n_q_heads;
-  if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
+  // grouped-query attention: pack the group's heads into common row tiles when the group size divides 128
+  const int group = a->n_q_heads / a->n_kv_heads;
+  const bool packed = group > 1 && (128 % group) == 0;
   TcParams p;
+  p.G = packed ? group : 1;
+  p.g_shift = 0;
+  while ((1 << p.g_shift) < p.G) ++p.g_shift;
+  p.HU = packed ? a->n_kv_heads : a->n_q_heads;
+  p.kv_div = packed ? 1 : group;
+  p.MT = (ctx->n_nodes * p.G + 127) / 128;
+  const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * p.HU * p.MT;
+  if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
   p.out = static_cast<__nv_bfloat16*>(a->out);
   p.ctx_len = a->d_ctx_len;
   p.anc = ctx->d_anc;
   p.part_o = ctx->d_attn_part_o;
   p.part_ml = ctx->d_attn_part_ml;
   p.flags = ctx->d_flags;
-  p.N = ctx->n_nodes; p.Hq = a->n_q_heads; p.Hkv = a->n_kv_heads; p.L = a->n_layers;
+  p.N = ctx->n_nodes; p.L = a->n_layers;
   p.os_b = a->o_stride[0]; p.os_h = a->o_stride[1]; p.os_t = a->o_stride[2]; p.os_l = a->layer_stride_o;
   const float scale = a->scale != 0.f ? a->scale : 1.0f / sqrtf(static_cast<float>(a->head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
   p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK, true);
   p.n_units = static_cast<int>(base * p.S);
-  magic_u32(static_cast<uint32_t>(a->n_q_heads / a->n_kv_heads), p.div_group);
+  magic_u32(static_cast<uint32_t>(p.MT), p.div_MT);
   magic_u32(static_cast<uint32_t>(p.S), p.div_S);
-  magic_u32(static_cast<uint32_t>(p.Hkv), p.div_Hkv);
+  magic_u32(static_cast<uint32_t>(p.HU), p.div_HU);
   magic_u32(static_cast<uint32_t>(p.L), p.div_L);
+  magic_u32(static_cast<uint32_t>(p.kv_div), p.div_kv);
 
   // Q is addressed as (dim, head, node, layer, sequence): in the usual [.., node, head, dim] layout the head
   // stride is the smaller one, and the tile (64 dims x 1 head x 128 nodes) lands in shared memory as 128 rows.
   CUtensorMap mq, mk, mv;
   const uint64_t qd[5] = {HD, (uint64_t)a->n_q_heads, (uint64_t)ctx->n_nodes, (uint64_t)a->n_layers, (uint64_t)ctx->batch};
   const int64_t qs[4] = {a->q_stride[1], a->q_stride[2], a->layer_stride_q, a->q_stride[0]};
-  const uint32_t qbox[5] = {64, 1, BK, 1, 1};
+  const uint32_t qbox[5] = {64, (uint32_t)p.G, (uint32_t)(128 / p.G), 1, 1};  // G heads x 128/G nodes = 128 rows
   const uint64_t kd[5] = {HD, (uint64_t)a->kv_rows, (uint64_t)a->n_kv_heads, (uint64_t)a->n_layers, (uint64_t)ctx->batch};
   const int64_t ks[4] = {a->kv_stride[2], a->kv_stride[1], a->layer_stride_kv, a->kv_stride[0]};
   const uint32_t kbox[5] = {64, BK, 1, 1, 1};
@@ -762,7 +820,8 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   const int grid = p.n_units < ctx->sm_count ? p.n_units : ctx->sm_count;
   tr_attn_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
   TR_CUDA_TRY(cudaGetLastError());
-  if (p.S > 1) tr_launch_attention_combine(ctx, a, p.S, s);
+  if (p.S > 1)
+    tr_attn_tc_combine_kernel<<<dim3(16, static_cast<unsigned>(base)), 256, 0, s>>>(p);
   TR_CUDA_TRY(cudaGetLastError());
   return TR_OK;
 }

@@ -255,6 +255,15 @@ def test_attention_gqa_and_batch_with_mixed_contexts(harness):
     _attention_case(harness, w, 1, splits=3)
 
 
+@pytest.mark.parametrize("hq,hkv", [(6, 2), (8, 1), (4, 2), (16, 2)])
+def test_attention_group_sizes(harness, hq, hkv):
+    """Grouped-query attention: group sizes that divide 128 share packed row tiles (2, 8; 8 heads of one KV head
+    fill five tiles with the 80-node tree), others (3) fall back to one tile per query head."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=hq, n_kv_heads=hkv, ctx=(150,))
+    _attention_case(harness, w, 1)
+    _attention_case(harness, w, 2, splits=2)
+
+
 def test_largest_tree_128_nodes_attention_and_loop(harness):
     # the maximum template size (ancestor masks are 128-bit; the attention tile has 128 query rows)
     w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], branching=(10, 10), n_nodes=128, n_q_heads=2, n_kv_heads=2,
