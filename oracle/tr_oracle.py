@@ -151,6 +151,31 @@ def argtopk(logits, k):
 
 
 # --------------------------------------------------------------------------
+# Output distribution from the last hidden states (Sec. 2.1: p = M(x); Sec. 5
+# notes that the model forward dominates a step).  The last linear layer of the
+# model followed directly by argtopk, so that the logits need not be stored.
+# --------------------------------------------------------------------------
+def lm_head_logits(hidden, weight):
+    """logits[i, v] = sum_h hidden[i, h] * weight[v, h], in float64 from the
+    given (bf16-valued) inputs; `weight` is [V, hidden] as a linear layer
+    stores it.  Definition written out with a library matrix product.
+    Pinned by: pure-Python integer dot products on a tiny case, one-hot hidden
+    rows (the logits are then a column of the weight), vocabulary permutation.
+    """
+    hidden = np.asarray(hidden, dtype=np.float64)
+    weight = np.asarray(weight, dtype=np.float64)
+    return hidden @ weight.T
+
+
+def lm_head_topk(hidden, weight, k):
+    """argtopk of the float32-rounded logits of every row (the comparison is
+    made in the kernel's precision, float32; the paper fixes none).  Returns
+    (indices [n, k], logits float64 [n, V])."""
+    logits = lm_head_logits(hidden, weight)
+    return argtopk(logits.astype(np.float32), k), logits
+
+
+# --------------------------------------------------------------------------
 # Verification (Sec. 2.2 "Guess and Verify", Sec. 3.3)
 # --------------------------------------------------------------------------
 def accept(S, argmax, parent):

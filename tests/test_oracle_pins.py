@@ -393,3 +393,64 @@ def test_commit_hand_example_and_gather_property():
     k = k0.copy(); v = v0.copy()
     orc.commit(k, v, 3, [], [0, 2, 3], [1, 2, 3])
     assert k[0, 3:6, 0].tolist() == [3, 5, 6]
+
+
+# ---------------------------------------------------------------------------
+# Output layer + argtopk (Sec. 2.1: p = M(x), x^0..x^{k-1} = argtopk(p))
+# ---------------------------------------------------------------------------
+def test_lm_head_bruteforce_small_integers():
+    """Pure-Python integer dot products and a (-value, index) sort on a tiny case full of ties."""
+    r = np.random.default_rng(5)
+    rows, H, V, k = 4, 6, 9, 5
+    hid = r.integers(-2, 3, size=(rows, H))
+    wt = r.integers(-2, 3, size=(V, H))
+    idx, logits = orc.lm_head_topk(hid, wt, k)
+    for i in range(rows):
+        dots = [sum(int(hid[i, h]) * int(wt[v, h]) for h in range(H)) for v in range(V)]
+        assert [float(d) for d in dots] == list(logits[i])
+        want = sorted(range(V), key=lambda v: (-dots[v], v))[:k]
+        assert list(idx[i]) == want
+    # a transposed weight or a sum over the wrong axis cannot pass: V != H here and wt is not symmetric
+
+
+def test_lm_head_one_hot_rows_select_weight_columns():
+    """hidden = e_h picks column h of the weight: the top-k is then the top-k of that column."""
+    r = np.random.default_rng(6)
+    V, H, k = 50, 8, 4
+    wt = r.standard_normal((V, H)).astype(np.float32)
+    hid = np.zeros((H, H), dtype=np.float32)
+    hid[np.arange(H), np.arange(H)] = 1.0
+    idx, logits = orc.lm_head_topk(hid, wt, k)
+    for h in range(H):
+        assert np.array_equal(logits[h], wt[:, h].astype(np.float64))
+        want = sorted(range(V), key=lambda v: (-float(wt[v, h]), v))[:k]
+        assert list(idx[h]) == want
+
+
+def test_lm_head_vocabulary_permutation_and_positive_scaling():
+    """Permuting the vocabulary rows of the weight permutes the indices; a positive scale of the hidden states
+    leaves them unchanged (tie-free random values)."""
+    r = np.random.default_rng(7)
+    rows, V, H, k = 5, 64, 16, 6
+    hid = r.standard_normal((rows, H)).astype(np.float32)
+    wt = r.standard_normal((V, H)).astype(np.float32)
+    idx, _ = orc.lm_head_topk(hid, wt, k)
+    perm = r.permutation(V)
+    idx_p, _ = orc.lm_head_topk(hid, wt[perm], k)
+    assert np.array_equal(perm[idx_p], idx)
+    idx_s, _ = orc.lm_head_topk(hid * 4.0, wt, k)
+    assert np.array_equal(idx_s, idx)
+
+
+def test_lm_head_synthetic_inputs():
+    w = synth.WORKLOADS["tiny"]
+    h1, w1 = synth.lm_head_inputs(w)
+    h2, w2 = synth.lm_head_inputs(w)
+    assert np.array_equal(h1, h2) and np.array_equal(w1, w2)
+    assert h1.shape == (w.batch * w.n_nodes, w.n_q_heads * w.head_dim) and w1.shape == (w.vocab, h1.shape[1])
+    hi, wi = synth.lm_head_inputs(w, kind="small-int")
+    fi, fw = synth.bf16_bits_to_f32(hi), synth.bf16_bits_to_f32(wi)
+    assert np.array_equal(fi, np.round(fi)) and np.abs(fi).max() <= 2 and np.abs(fw).max() <= 3
+    # small-integer inputs: the logits are exact integers, identical in float32 and float64
+    _, logits = orc.lm_head_topk(fi, fw, w.k)
+    assert np.array_equal(logits, np.round(logits)) and np.array_equal(logits.astype(np.float32).astype(np.float64), logits)
