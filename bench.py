@@ -160,6 +160,40 @@ def run_reference(args, w):
 
 
 # ---------------------------------------------------------------------------------------------------
+def measure_lm_head(torch, tr, dw, w, dev, reps=20):
+    """The output layer fused with argtopk (not part of the timed step, whose logits come from the toy model): one
+    pass over a random bf16 weight [V, hidden] for the step's batch * N rows, as a CUDA graph replayed `reps` times.
+    The weight (hundreds of MB) is larger than L2, so every replay streams it from HBM."""
+    H = w.n_q_heads * w.head_dim
+    rows = w.batch * w.n_nodes
+    g = torch.Generator(device=dev).manual_seed(w.seed & 0x7FFFFFFF)
+    d_h = torch.randn(rows, H, device=dev, generator=g).to(torch.bfloat16)
+    d_w = torch.randn(w.vocab, H, device=dev, generator=g).to(torch.bfloat16)
+    idx = torch.zeros(rows, w.k, dtype=torch.int32, device=dev)
+    s = torch.cuda.Stream(dev)
+    graph = torch.cuda.CUDAGraph()
+    tr.tr_lm_head_topk(dw.ctx, d_h, d_w, idx)
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s):
+        with torch.cuda.graph(graph, stream=s):
+            tr.tr_lm_head_topk(dw.ctx, d_h, d_w, idx, stream=s)
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        graph.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) / reps * 1000.0
+    passes = (rows + 127) // 128                               # one pass over the weight per 128 rows
+    byts = passes * w.vocab * H * 2 + rows * H * 2 + rows * w.k * 4
+    return {"us": us, "bound": "hbm", "achieved": byts / us / 1e3, "unit": "GB/s", "algorithmic_bytes": byts,
+            "rows": rows, "hidden": H, "vocab": w.vocab, "gpu_launches": passes + 1,
+            "device_flags": tr.tr_device_flags(dw.ctx)}
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -290,6 +324,8 @@ def run_ours(args, w):
     e2e_ms = (time.perf_counter() - t0) * 1000.0
     e2e = replicas.aggregate(e2e_ms, Ke, device=dev if world > 1 else "cpu")
 
+    lm = measure_lm_head(torch, tr, dw, w, dev) if rank == 0 else None
+
     if rank == 0:
         peak, peak_src = load_peaks()
         ab = algorithmic_bytes(w, dw.L)
@@ -322,6 +358,7 @@ def run_ours(args, w):
             "gpu_launches": dw.kernels_per_step() * K,
             "clocks": clocks,
             "mean_new_tokens_per_step": n_new_sum / (B * n_stat),
+            "next_rows": {"lm_head_topk": dict(lm, frac=lm["achieved"] / peak, peak=peak)},
             "device_flags": flags,
         }
         print(json.dumps(line), flush=True)

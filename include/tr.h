@@ -145,7 +145,34 @@ typedef struct {
 } tr_step_out;
 tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const int32_t* d_tree, const tr_step_out* out,
                            void* stream);
-int32_t tr_max_new_tokens(const tr_ctx* ctx);
+int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appendix: maximum acceptance length) */
+
+/*
+ * The same step from a top-k that is already on the device (for example from tr_lm_head_topk): everything
+ * tr_verify_update does after its argtopk.  out->d_topk_idx [batch, N, k] is an INPUT here (indices in [0, V),
+ * column 0 the argmax); the other members of `out` are written as by tr_verify_update.
+ */
+tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream);
+
+/*
+ * Output layer fused with argtopk (Sec. 2.1: p = M(x), x^0..x^{k-1} = argtopk(p); Sec. 5.4: the forward pass is most of
+ * a step).  For the rows = batch * N tree nodes,
+ *     logits[r, v] = sum_h hidden[r, h] * weight[v, h]      bf16 inputs, fp32 accumulation on the tensor cores
+ *     topk[r, :]   = indices of the k largest logits of row r, largest first, equal values by lower index
+ * and the [rows, V] logits are never written to memory: every CTA streams one slice of the weight once and keeps the
+ * per-row candidates of its slice; a second small kernel merges the slices.  The comparison is made on the fp32
+ * accumulators; their summation order is the hardware's, so two logits closer than fp32 rounding of a length-hidden
+ * dot product may come out in either order (inputs whose products and sums are exact give exact results).
+ * DEVICE in : d_hidden [rows, hidden_dim] bf16, row stride hidden_stride elements; d_weight [V, hidden_dim] bf16 (the
+ *             layout of a linear layer's weight), row stride weight_stride elements.  Both 16-byte aligned, strides
+ *             multiples of 8 and >= hidden_dim, hidden_dim a multiple of 8 (else TR_ERR_INVALID_ARG).  No NaN.
+ * DEVICE out: d_topk_idx [rows, k] int32; d_topk_val [rows, k] fp32 (the accumulated logits at those indices) or NULL.
+ * Rows are processed in groups of 128, each group with its own pass over the weight.  Allocates nothing, reads
+ * nothing back, does not synchronise; uses scratch of the context (not re-entrant per context).
+ */
+tr_status tr_lm_head_topk(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,
+                          int64_t weight_stride, int32_t hidden_dim, int32_t* d_topk_idx, float* d_topk_val,
+                          void* stream);
 
 /*
  * Update-rule variants the paper compares (Sec. 5.2 "Update Strategies" and "Effect of Rejected Tokens"; Appendix
@@ -160,7 +187,7 @@ int32_t tr_max_new_tokens(const tr_ctx* ctx);
 #define TR_UPDATE_FIRST 1
 #define TR_UPDATE_ALL_DRAFT 0
 #define TR_UPDATE_ONLY_ACCEPTED 1
-tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope); /* depth of the template + 1 (Appendix: maximum acceptance length) */
+tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope);
 
 /*
  * Commit the accepted path (Sec. 5.4: a step ends by "updating the matrix, input tokens, and key-value cache").

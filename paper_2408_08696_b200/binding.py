@@ -91,6 +91,9 @@ lib.tr_step_host.argtypes = [C.c_void_p, C.POINTER(tr_attn_args), C.POINTER(tr_s
 lib.tr_commit.argtypes = [C.c_void_p, C.POINTER(tr_commit_args), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 lib.tr_topk_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
 lib.tr_topk_noalloc_limits.argtypes = [_P32, _P32]
+lib.tr_verify_update_topk.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(tr_step_out), C.c_void_p]
+lib.tr_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p,
+                                C.c_void_p, C.c_void_p]
 lib_synth.trs_patch_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
                                        C.c_int32, C.c_int32, C.c_void_p]
 
@@ -241,6 +244,31 @@ def tr_verify_update(ctx, d_logits, d_tree, out_struct, stream=None):
     _check(lib.tr_verify_update(ctx.handle, _dev(d_logits, torch.float32, "d_logits"),
                                 _dev(d_tree, torch.int32, "d_tree"), C.byref(out_struct), _stream(stream)),
            "tr_verify_update")
+
+
+def tr_verify_update_topk(ctx, d_tree, out_struct, stream=None):
+    """The step from a top-k already in out_struct.d_topk_idx (for example written by tr_lm_head_topk)."""
+    _check(lib.tr_verify_update_topk(ctx.handle, _dev(d_tree, torch.int32, "d_tree"), C.byref(out_struct),
+                                     _stream(stream)), "tr_verify_update_topk")
+
+
+def tr_lm_head_topk(ctx, d_hidden, d_weight, d_topk_idx, d_topk_val=None, stream=None):
+    """d_hidden bf16 [batch * N, hidden], d_weight bf16 [V, hidden] (inner dimension contiguous);
+    d_topk_idx int32 [batch * N, k] (any shape with that many elements), d_topk_val float32 likewise or None."""
+    rows = ctx.batch * ctx.n_nodes
+    if d_hidden.dim() != 2 or d_weight.dim() != 2 or d_hidden.shape[0] != rows or d_weight.shape[0] != ctx.vocab \
+            or d_hidden.shape[1] != d_weight.shape[1] or d_hidden.stride(1) != 1 or d_weight.stride(1) != 1:
+        raise ValueError("d_hidden must be [batch*N, hidden] and d_weight [V, hidden], inner dimension contiguous")
+    if d_topk_idx.numel() != rows * ctx.k or not d_topk_idx.is_contiguous():
+        raise ValueError("d_topk_idx must be contiguous with batch*N*k elements")
+    val = None
+    if d_topk_val is not None:
+        if d_topk_val.numel() != rows * ctx.k or not d_topk_val.is_contiguous():
+            raise ValueError("d_topk_val must be contiguous with batch*N*k elements")
+        val = _dev(d_topk_val, torch.float32, "d_topk_val")
+    _check(lib.tr_lm_head_topk(ctx.handle, _dev(d_hidden, torch.bfloat16, "d_hidden"), d_hidden.stride(0),
+                               _dev(d_weight, torch.bfloat16, "d_weight"), d_weight.stride(0), d_hidden.shape[1],
+                               _dev(d_topk_idx, torch.int32, "d_topk_idx"), val, _stream(stream)), "tr_lm_head_topk")
 
 
 def make_commit_args(ctx, k_cache, v_cache, d_ctx_len, d_tokens, d_n_tokens):

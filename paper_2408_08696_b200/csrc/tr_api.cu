@@ -61,6 +61,7 @@ static tr_status free_all(tr_ctx* c) {
   cudaFree(c->d_topk_part);
   cudaFree(c->d_topk_ticket);
   cudaFree(c->d_seq_ticket);
+  cudaFree(c->d_lm_part);
   cudaFree(c->d_attn_part_o);
   cudaFree(c->d_attn_part_ml);
   cudaFree(c->d_flags);
@@ -141,6 +142,8 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaMemset(c->d_topk_ticket, 0, sizeof(unsigned int) * rows));
   TR_INIT_TRY(cudaMalloc(&c->d_seq_ticket, sizeof(unsigned int) * batch));
   TR_INIT_TRY(cudaMemset(c->d_seq_ticket, 0, sizeof(unsigned int) * batch));
+  c->lm_parts_cap = 2 * c->sm_count;  // two lists per CTA
+  TR_INIT_TRY(cudaMalloc(&c->d_lm_part, sizeof(unsigned long long) * rows * c->lm_parts_cap * k));
 
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_o, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 128));
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_ml, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 2));
@@ -151,6 +154,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   {
     tr_status st = tr_attention_mma_setup();
     if (st == TR_OK) st = tr_attention_tc_setup();
+    if (st == TR_OK) st = tr_lm_head_setup();
     const char* force = getenv("TR_ATTN_FORCE_MMA");
     c->force_mma = force && force[0] == '1';
     if (st != TR_OK) {
@@ -232,6 +236,27 @@ extern "C" tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const 
   tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s);
   if (st != TR_OK) return st;
   return tr_launch_tail(ctx, d_tree, out, s);
+}
+
+extern "C" tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream) {
+  if (!ctx || !d_tree || !out) return TR_ERR_INVALID_ARG;
+  if (!out->d_topk_idx || !out->d_n_new || !out->d_acc_nodes || !out->d_out_tokens || !out->d_next_root ||
+      !out->d_next_tree)
+    return TR_ERR_INVALID_ARG;
+  return tr_launch_tail(ctx, d_tree, out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" tr_status tr_lm_head_topk(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,
+                                     int64_t weight_stride, int32_t hidden_dim, int32_t* d_topk_idx, float* d_topk_val,
+                                     void* stream) {
+  if (!ctx || !d_hidden || !d_weight || !d_topk_idx) return TR_ERR_INVALID_ARG;
+  if (hidden_dim < 8 || (hidden_dim % 8) != 0) return TR_ERR_INVALID_ARG;
+  if (hidden_stride < hidden_dim || weight_stride < hidden_dim || (hidden_stride % 8) != 0 || (weight_stride % 8) != 0)
+    return TR_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(d_hidden) & 15) != 0 || (reinterpret_cast<uintptr_t>(d_weight) & 15) != 0)
+    return TR_ERR_INVALID_ARG;
+  return tr_launch_lm_head(ctx, d_hidden, hidden_stride, d_weight, weight_stride, hidden_dim, d_topk_idx, d_topk_val,
+                           static_cast<cudaStream_t>(stream));
 }
 
 static tr_status check_attn_args(const tr_ctx* ctx, const tr_attn_args* a) {

@@ -44,6 +44,8 @@ struct tr_ctx {
   unsigned int* d_topk_ticket = nullptr;      // [batch*N]
   unsigned int* d_seq_ticket = nullptr;       // [batch]: CTAs of a sequence that passed tr_commit's read phase
   int topk_segs = 0;
+  unsigned long long* d_lm_part = nullptr;    // [batch*N][lm_parts_cap][k] per-CTA lists of tr_lm_head_topk
+  int lm_parts_cap = 0;
   float* d_attn_part_o = nullptr;   // [slots][128][128]
   float* d_attn_part_ml = nullptr;  // [slots][128][2]
   uint32_t* d_flags = nullptr;
@@ -83,4 +85,7 @@ tr_status tr_attention_mma_setup();
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_tc_setup();
 void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
+tr_status tr_lm_head_setup();
+tr_status tr_launch_lm_head(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,
+                            int64_t weight_stride, int hidden_dim, int32_t* d_topk_idx, float* d_topk_val, cudaStream_t s);
 int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys, bool fill_once);
