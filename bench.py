@@ -385,10 +385,19 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
     ap.add_argument("--profile", action="store_true",
                     help="only warm up and replay the step graph K times (for ncu); prints no bench line")
+    ap.add_argument("--lm-head-only", action="store_true",
+                    help="only time the output layer fused with argtopk (for ncu); prints its figures, no bench line")
     args = ap.parse_args()
     from paper_2408_08696_b200 import synth
     w = synth.WORKLOADS[args.workload]
-    if args.impl == "reference":
+    if args.lm_head_only:
+        import torch
+        from paper_2408_08696_b200 import binding as tr
+        from paper_2408_08696_b200 import harness
+        dw = harness.DeviceWorkload(w, with_attention=False)
+        print(json.dumps({"lm_head_topk": measure_lm_head(torch, tr, dw, w, dw.dev, reps=5), "workload": w.name}))
+        dw.close()
+    elif args.impl == "reference":
         run_reference(args, w)
     else:
         run_ours(args, w)

@@ -2,8 +2,8 @@
 // warp-specialised flash-decoding kernel.
 //
 //   warps 0..3  epilogue: thread r normalises output row r out of TMEM and stores it, off the softmax warps' path
-//   warp 8      TMA producer: Q tile (double-buffered) and a ring of 32 KB K / V tiles (128 keys x 128 dims, bf16,
-//               128-byte swizzle), one mbarrier per ring slot
+//   warp 8      TMA producer: Q tile (double-buffered, or single with one more ring slot: kQSingle) and a ring of
+//               32 KB K / V tiles (128 keys x 128 dims, bf16, 128-byte swizzle), one mbarrier per ring slot
 //   warp 9      MMA issuer: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM) and
 //               O += P V (P read from TMEM, V as an MN-major shared-memory operand); owns the TMEM allocation
 //   warps 4..7  softmax: thread r owns query row r (= TMEM lane r): loads its S row, applies the ancestor mask
@@ -41,7 +41,8 @@ namespace {
 
 constexpr int BK = 128;          // keys per tile
 constexpr int HD = 128;          // head_dim
-constexpr int NST = 5;           // ring slots (K and V tiles alternate)
+constexpr int NST_MAX = 6;       // ring slots (K and V tiles alternate): 5 beside a double-buffered Q tile, 6 beside a
+                                 // single one (kQSingle: long units, where the Q reload between units is negligible)
 constexpr int TILE_BYTES = BK * HD * 2;       // 32 KB
 constexpr int HALF_BYTES = TILE_BYTES / 2;    // one TMA box: 64 dims x 128 rows
 constexpr int NTHREADS = 384;       // warps 0-3 epilogue, 4-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle
@@ -68,9 +69,8 @@ struct TcParams {
 
 // shared memory map (offsets from a 1024-byte aligned base)
 constexpr int SM_Q = 0;                               // 2 x 32 KB
-constexpr int SM_RING = 2 * TILE_BYTES;               // NST x 32 KB
-constexpr int SM_BAR = SM_RING + NST * TILE_BYTES;    // mbarriers
-constexpr int BAR_FULL = 0, BAR_EMPTY = NST, BAR_QFULL = 2 * NST, BAR_QEMPTY = BAR_QFULL + 2,
+constexpr int SM_BAR = 7 * TILE_BYTES;                // Q tile(s) + ring = 7 x 32 KB, then the mbarriers
+constexpr int BAR_FULL = 0, BAR_EMPTY = NST_MAX, BAR_QFULL = 2 * NST_MAX, BAR_QEMPTY = BAR_QFULL + 2,
               BAR_SFULL = BAR_QEMPTY + 2, BAR_PFULL = BAR_SFULL + 2, BAR_PVDONE = BAR_PFULL + 2,
               BAR_OFREE = BAR_PVDONE + 2, BAR_OREADY = BAR_OFREE + 2, BAR_LFULL = BAR_OREADY + 2,
               BAR_COUNT = BAR_LFULL + 2;
@@ -172,6 +172,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+template <bool kQSingle>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -182,6 +183,8 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (threadIdx.x == 0) atomicOr(p.flags, TR_FLAG_WAIT_TIMEOUT);
     return;
   }
+  constexpr int NST = kQSingle ? 6 : 5;
+  constexpr int SM_RING = (kQSingle ? 1 : 2) * TILE_BYTES;
   const uint32_t bars = base + SM_BAR;
   volatile uint32_t* s_tmem = reinterpret_cast<volatile uint32_t*>(base_ptr + SM_MISC);
   volatile uint32_t* s_abort = s_tmem + 1;
@@ -195,7 +198,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   }
 
   if (tid == 0) {
-    for (int i = 0; i < NST; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
+    for (int i = 0; i < NST_MAX; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_QFULL + i), 1);
       mbar_init(bar(BAR_QEMPTY + i), 1);
@@ -233,9 +236,9 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
         const Unit x = decode_unit(p, u, s_ctx);
         if (x.t0 >= x.t1) continue;
-        const uint32_t qb = ui & 1u;
+        const uint32_t qb = kQSingle ? 0u : (ui & 1u);
         USTAMP(0, ui, 0)
-        ok = mbar_wait(bar(BAR_QEMPTY + qb), ((ui >> 1) & 1u) ^ 1u, s_abort);
+        ok = mbar_wait(bar(BAR_QEMPTY + qb), ((kQSingle ? ui : (ui >> 1)) & 1u) ^ 1u, s_abort);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_QFULL + qb), TILE_BYTES);
         tma_load_5d(base + SM_Q + qb * TILE_BYTES, &map_q, bar(BAR_QFULL + qb), 0, x.h0, x.node0, x.layer, x.b);
@@ -274,9 +277,9 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       kc.init(p, s_ctx);
       vc.init(p, s_ctx);
       auto issue_qk = [&]() -> bool {  // S = Q K^T of the tile under kc
-        const uint32_t sb = kc.g & 1u, c = 2u * kc.g, slot = c % NST, qb = kc.ui & 1u;
+        const uint32_t sb = kc.g & 1u, c = 2u * kc.g, slot = c % NST, qb = kQSingle ? 0u : (kc.ui & 1u);
         bool w = true;
-        if (kc.j == 0) WAITACC(4, w = mbar_wait(bar(BAR_QFULL + qb), (kc.ui >> 1) & 1u, s_abort))
+        if (kc.j == 0) WAITACC(4, w = mbar_wait(bar(BAR_QFULL + qb), (kQSingle ? kc.ui : (kc.ui >> 1)) & 1u, s_abort))
         if (!w) return false;
         // the S/P buffer is free once the PV of tile g-2 has completed
         WAITACC(3, w = mbar_wait(bar(BAR_PVDONE + sb), ((kc.g >> 1) & 1u) ^ 1u, s_abort))
@@ -615,7 +618,8 @@ __global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams 
 }  // namespace
 
 tr_status tr_attention_tc_setup() {
-  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
   return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
 }
 
@@ -674,7 +678,12 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
       !encode_map(&mv, a->v_cache, kd, ks, kbox))
     return TR_ERR_UNSUPPORTED;
   const int grid = p.n_units < ctx->sm_count ? p.n_units : ctx->sm_count;
-  tr_attn_tc_kernel<<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+  // Grouped-query shapes (several row tiles per KV head, long units, K/V re-read from L2): one Q buffer and a sixth
+  // ring slot; otherwise Q is double-buffered so that short units overlap their Q load.
+  if (p.MT > 1)
+    tr_attn_tc_kernel<true><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+  else
+    tr_attn_tc_kernel<false><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
   TR_CUDA_TRY(cudaGetLastError());
   if (p.S > 1)
     tr_attn_tc_combine_kernel<<<dim3(16, static_cast<unsigned>(base)), 256, 0, s>>>(p);

@@ -275,6 +275,21 @@ def test_largest_tree_128_nodes_attention_and_loop(harness):
     _run_loop(harness, w, 6)
 
 
+@pytest.mark.parametrize("branching,n_nodes,k,boost", [
+    ((1,) * 24, 25, 8, 9.0),                 # a chain: depth 24, accepted paths get long with a strong toy model
+    ((2,) * 6, 127, 8, 4.0),                 # full binary tree, depth 6
+    ((16,), 17, 16, 4.0),                    # a star: one level, every rank up to k - 1 = 15
+    ((8, 4, 3, 2, 2, 1, 1, 1, 1, 1), 110, 8, 6.0),   # the default shape made deeper (Fig. 3b's knob)
+    ((12, 6, 3, 1), 120, 12, 3.0),           # ... and broader (Fig. 3a's knob)
+])
+def test_loop_template_breadth_and_depth_sweep(harness, branching, n_nodes, k, boost):
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], branching=branching, n_nodes=n_nodes, k=k, boost=boost,
+                            vocab=2000)
+    mat = _run_loop(harness, w, 20)
+    parent, _ = orc.template_from_branching(branching, n_nodes)
+    assert 1.0 <= mat <= max(orc.node_depth(parent)) + 1          # Appendix: at most depth + 1 tokens per step
+
+
 def test_attention_single_node_tree(harness):
     w = dataclasses.replace(synth.WORKLOADS["tiny"], n_nodes=1, branching=(1,), ctx=(50,))
     _attention_case(harness, w, 1)
