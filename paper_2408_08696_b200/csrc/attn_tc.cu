@@ -172,7 +172,7 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
-template <bool kQSingle>
+template <bool kQSingle, bool kPdl>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const TcParams p) {
@@ -192,10 +192,11 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   int* s_ctx = reinterpret_cast<int*>(base_ptr + SM_CTX);
-  {
+  auto stage_ctx_len = [&]() {
     const int nb = p.n_units / (p.L * p.HU * p.S * p.MT);  // sequences
     if (tid >= 64 && tid - 64 < CTX_CACHE && tid - 64 < nb) s_ctx[tid - 64] = p.ctx_len[tid - 64];
-  }
+  };
+  if (!kPdl) stage_ctx_len();
 
   if (tid == 0) {
     for (int i = 0; i < NST_MAX; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
@@ -217,6 +218,12 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + SM_MISC), "r"(512u)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  if (kPdl) {
+    // launched with programmatic dependent launch (short launches only): everything above touches only this CTA's
+    // shared memory and TMEM; the context lengths, Q/K/V and the partial buffers belong to whatever ran before
+    tr_grid_dependency_wait();
+    stage_ctx_len();
   }
   tc_fence_before();
   __syncthreads();
@@ -582,6 +589,7 @@ bool encode_map(CUtensorMap* m, const void* ptr, const uint64_t (&dims)[5], cons
 // One CTA per (8 tile rows, tile); 32 lanes x float4 cover the 128 dims of a row.  Slots are numbered like the
 // units: (((b, layer, head unit), split), tile).
 __global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams p) {
+  tr_grid_dependency_wait();  // launched with programmatic dependent launch: the partials come from the kernel before
   const int r = blockIdx.x * 8 + (threadIdx.x >> 5);  // row of the tile
   const int d = (threadIdx.x & 31) * 4;
   const uint32_t t = blockIdx.y;                        // (b, layer, head unit, tile)
@@ -618,8 +626,9 @@ __global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams 
 }  // namespace
 
 tr_status tr_attention_tc_setup() {
-  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
   return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
 }
 
@@ -681,12 +690,16 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   // Grouped-query shapes (several row tiles per KV head, long units, K/V re-read from L2): one Q buffer and a sixth
   // ring slot; otherwise Q is double-buffered so that short units overlap their Q load.
   if (p.MT > 1)
-    tr_attn_tc_kernel<true><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+    tr_attn_tc_kernel<true, false><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+  else if (p.S > 1)
+    // a short launch (fewer units than SMs, split along the keys) between other short kernels, typically one layer's
+    // attention: programmatic dependent launch hides its launch latency (503 -> 475 us for 32 per-layer launches at
+    // the 7B shape).  Long launches gain nothing from it and measured about 1.5 % slower.
+    TR_CUDA_TRY(tr_launch_pdl(tr_attn_tc_kernel<false, true>, dim3(grid), dim3(NTHREADS), SMEM_BYTES, s, mq, mk, mv, p));
   else
-    tr_attn_tc_kernel<false><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+    tr_attn_tc_kernel<false, false><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
   TR_CUDA_TRY(cudaGetLastError());
   if (p.S > 1)
-    tr_attn_tc_combine_kernel<<<dim3(16, static_cast<unsigned>(base)), 256, 0, s>>>(p);
-  TR_CUDA_TRY(cudaGetLastError());
+    TR_CUDA_TRY(tr_launch_pdl(tr_attn_tc_combine_kernel, dim3(16, static_cast<unsigned>(base)), dim3(256), 0, s, p));
   return TR_OK;
 }
