@@ -29,6 +29,8 @@ constexpr int LM_MAX_STAGES = 8;
 constexpr int LM_A_BYTES = 128 * LM_BK * 2;     // 16 KB: 128 query rows
 constexpr int LM_RING_BYTES = 224 * 1024;       // stages of LM_A_BYTES + NC * 128 bytes each
 constexpr int LM_THREADS = 320;
+constexpr int LM_MAX_NC = 256;                  // widest chunk = the MMA's largest N (narrower chunks hide more
+                                                // epilogues but re-read the hidden states more often: measured slower)
 constexpr int LM_SM_BAR = LM_RING_BYTES;
 constexpr int LM_BAR_FULL = 0, LM_BAR_EMPTY = LM_MAX_STAGES, LM_BAR_ACC_FULL = 2 * LM_MAX_STAGES,
               LM_BAR_ACC_EMPTY = LM_BAR_ACC_FULL + 2, LM_BAR_COUNT = LM_BAR_ACC_EMPTY + 2;
@@ -344,7 +346,7 @@ static void lm_partition(const tr_ctx* ctx, LmParams* p, int* n_cta) {
   w = (w + 15) / 16 * 16;
   p->cols_per_cta = w;
   *n_cta = (ctx->vocab + w - 1) / w;
-  p->n_main = (w + 255) / 256;
+  p->n_main = (w + LM_MAX_NC - 1) / LM_MAX_NC;
   p->NC = ((w + p->n_main - 1) / p->n_main + 15) / 16 * 16;
   const int stage = LM_A_BYTES + p->NC * LM_BK * 2;
   p->nstage = LM_RING_BYTES / stage < LM_MAX_STAGES ? LM_RING_BYTES / stage : LM_MAX_STAGES;
