@@ -234,7 +234,9 @@ tr_status tr_device_flags(tr_ctx* ctx, uint32_t* host_flags);
  *           current tree (updated in place to the next tree); d_out as in tr_verify_update.
  * HOST out: h_out [batch, L, N, Hq, D] bf16; h_n_new [batch]; h_out_tokens [batch, depth_max+1];
  *           h_next_tree [batch, N].
- * Synchronises `stream` before returning.
+ * The layers are independent, so the copies are pipelined against the attention launches over groups of layers on
+ * two internal copy streams of the context (inputs of group g+1 and outputs of group g-1 move while group g
+ * computes); everything is ordered after the work already queued on `stream`, which is synchronised before returning.
  */
 typedef struct {
   const void* h_q;

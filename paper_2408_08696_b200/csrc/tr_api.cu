@@ -62,6 +62,13 @@ static tr_status free_all(tr_ctx* c) {
   cudaFree(c->d_topk_ticket);
   cudaFree(c->d_seq_ticket);
   cudaFree(c->d_lm_part);
+  if (c->io_in) cudaStreamDestroy(c->io_in);
+  if (c->io_out) cudaStreamDestroy(c->io_out);
+  for (cudaEvent_t e : {c->ev_start, c->ev_logits, c->ev_out}) if (e) cudaEventDestroy(e);
+  for (int g = 0; g < TR_IO_GROUPS; ++g) {
+    if (c->ev_in[g]) cudaEventDestroy(c->ev_in[g]);
+    if (c->ev_attn[g]) cudaEventDestroy(c->ev_attn[g]);
+  }
   cudaFree(c->d_attn_part_o);
   cudaFree(c->d_attn_part_ml);
   cudaFree(c->d_flags);
@@ -147,6 +154,16 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
 
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_o, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 128));
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_ml, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 2));
+  // streams and events of tr_step_host's copy pipeline
+  TR_INIT_TRY(cudaStreamCreateWithFlags(&c->io_in, cudaStreamNonBlocking));
+  TR_INIT_TRY(cudaStreamCreateWithFlags(&c->io_out, cudaStreamNonBlocking));
+  TR_INIT_TRY(cudaEventCreateWithFlags(&c->ev_start, cudaEventDisableTiming));
+  TR_INIT_TRY(cudaEventCreateWithFlags(&c->ev_logits, cudaEventDisableTiming));
+  TR_INIT_TRY(cudaEventCreateWithFlags(&c->ev_out, cudaEventDisableTiming));
+  for (int g = 0; g < TR_IO_GROUPS; ++g) {
+    TR_INIT_TRY(cudaEventCreateWithFlags(&c->ev_in[g], cudaEventDisableTiming));
+    TR_INIT_TRY(cudaEventCreateWithFlags(&c->ev_attn[g], cudaEventDisableTiming));
+  }
   TR_INIT_TRY(cudaMalloc(&c->d_flags, sizeof(uint32_t)));
   TR_INIT_TRY(cudaMemset(c->d_flags, 0, sizeof(uint32_t)));
   TR_INIT_TRY(cudaDeviceSynchronize());
@@ -315,43 +332,80 @@ extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_s
   const int B = ctx->batch, N = ctx->n_nodes, L = a->n_layers, D = a->head_dim;
   const size_t esz = sizeof(__nv_bfloat16);
   // queries: the staging tensor must be dense [B, L, N, Hq, D]
-  const size_t q_elems = static_cast<size_t>(B) * L * N * a->n_q_heads * D;
   if (a->q_stride[2] != (int64_t)a->n_q_heads * D || a->q_stride[1] != D ||
       a->layer_stride_q != (int64_t)N * a->n_q_heads * D || a->q_stride[0] != (int64_t)L * N * a->n_q_heads * D ||
       a->o_stride[2] != a->q_stride[2] || a->o_stride[1] != D || a->layer_stride_o != a->layer_stride_q ||
       a->o_stride[0] != a->q_stride[0])
     return TR_ERR_INVALID_ARG;
-  TR_CUDA_TRY(cudaMemcpyAsync(const_cast<void*>(a->q), io->h_q, q_elems * esz, cudaMemcpyHostToDevice, s));
-  // this step's tree K/V rows go behind each sequence's prefix: one strided copy per (sequence, layer)
-  for (int b = 0; b < B; ++b) {
-    const int C = io->h_ctx_len[b];
-    if (C < 0 || C > a->max_ctx) return TR_ERR_INVALID_ARG;
-    for (int l = 0; l < L; ++l) {
-      const size_t src_off = (static_cast<size_t>(b) * L + l) * a->n_kv_heads * N * D;
-      const size_t dst_off = b * a->kv_stride[0] + l * a->layer_stride_kv + static_cast<size_t>(C) * a->kv_stride[2];
-      if (a->kv_stride[2] != D) return TR_ERR_UNSUPPORTED;
-      // rows of one head are contiguous (N*D elements); heads are kv_stride[1] apart
-      TR_CUDA_TRY(cudaMemcpy2DAsync((__nv_bfloat16*)a->k_cache + dst_off, a->kv_stride[1] * esz,
-                                    (const __nv_bfloat16*)io->h_tree_k + src_off, (size_t)N * D * esz,
-                                    (size_t)N * D * esz, a->n_kv_heads, cudaMemcpyHostToDevice, s));
-      TR_CUDA_TRY(cudaMemcpy2DAsync((__nv_bfloat16*)a->v_cache + dst_off, a->kv_stride[1] * esz,
-                                    (const __nv_bfloat16*)io->h_tree_v + src_off, (size_t)N * D * esz,
-                                    (size_t)N * D * esz, a->n_kv_heads, cudaMemcpyHostToDevice, s));
+  if (a->kv_stride[2] != D) return TR_ERR_UNSUPPORTED;
+  for (int bq = 0; bq < B; ++bq)
+    if (io->h_ctx_len[bq] < 0 || io->h_ctx_len[bq] > a->max_ctx) return TR_ERR_INVALID_ARG;
+  // The layers are independent, so the step is pipelined over groups of layers on three streams: while group g's
+  // attention runs, group g+1's inputs are on their way in and group g-1's output is on its way out (PCIe carries
+  // both directions at once).  Host -> device on io_in, kernels on the caller's stream, device -> host on io_out.
+  const int G = L < TR_IO_GROUPS ? L : TR_IO_GROUPS;
+  TR_CUDA_TRY(cudaEventRecord(ctx->ev_start, s));  // whatever the caller queued before comes first on all three
+  TR_CUDA_TRY(cudaStreamWaitEvent(ctx->io_in, ctx->ev_start, 0));
+  TR_CUDA_TRY(cudaStreamWaitEvent(ctx->io_out, ctx->ev_start, 0));
+  const size_t q_layer = static_cast<size_t>(N) * a->n_q_heads * D;  // elements of one (sequence, layer) of Q / out
+  for (int g = 0; g < G; ++g) {
+    const int l0 = static_cast<int>(static_cast<int64_t>(L) * g / G), l1 = static_cast<int>(static_cast<int64_t>(L) * (g + 1) / G);
+    const int nl = l1 - l0;
+    for (int b = 0; b < B; ++b) {
+      const int C = io->h_ctx_len[b];
+      const size_t q_off = (static_cast<size_t>(b) * L + l0) * q_layer;
+      TR_CUDA_TRY(cudaMemcpyAsync((__nv_bfloat16*)a->q + q_off, (const __nv_bfloat16*)io->h_q + q_off, nl * q_layer * esz,
+                                  cudaMemcpyHostToDevice, ctx->io_in));
+      // this step's tree K/V rows go behind the sequence's prefix: the N rows of one head are contiguous (N*D
+      // elements) and heads are kv_stride[1] apart; when the layers are Hkv heads apart as well (a dense cache), the
+      // group's (layer, head) pairs form one run of equally spaced rows and a single strided copy moves them all
+      const bool dense = a->layer_stride_kv == static_cast<int64_t>(a->n_kv_heads) * a->kv_stride[1];
+      const int ncopies = dense ? 1 : nl;
+      for (int i = 0; i < ncopies; ++i) {
+        const int l = l0 + i;
+        const size_t src_off = (static_cast<size_t>(b) * L + l) * a->n_kv_heads * N * D;
+        const size_t dst_off = b * a->kv_stride[0] + l * a->layer_stride_kv + static_cast<size_t>(C) * a->kv_stride[2];
+        const size_t height = static_cast<size_t>(dense ? nl : 1) * a->n_kv_heads;
+        TR_CUDA_TRY(cudaMemcpy2DAsync((__nv_bfloat16*)a->k_cache + dst_off, a->kv_stride[1] * esz,
+                                      (const __nv_bfloat16*)io->h_tree_k + src_off, (size_t)N * D * esz,
+                                      (size_t)N * D * esz, height, cudaMemcpyHostToDevice, ctx->io_in));
+        TR_CUDA_TRY(cudaMemcpy2DAsync((__nv_bfloat16*)a->v_cache + dst_off, a->kv_stride[1] * esz,
+                                      (const __nv_bfloat16*)io->h_tree_v + src_off, (size_t)N * D * esz,
+                                      (size_t)N * D * esz, height, cudaMemcpyHostToDevice, ctx->io_in));
+      }
+    }
+    TR_CUDA_TRY(cudaEventRecord(ctx->ev_in[g], ctx->io_in));
+    TR_CUDA_TRY(cudaStreamWaitEvent(s, ctx->ev_in[g], 0));
+    tr_attn_args ag = *a;
+    ag.q = (const __nv_bfloat16*)a->q + l0 * a->layer_stride_q;
+    ag.k_cache = (const __nv_bfloat16*)a->k_cache + l0 * a->layer_stride_kv;
+    ag.v_cache = (const __nv_bfloat16*)a->v_cache + l0 * a->layer_stride_kv;
+    ag.out = (__nv_bfloat16*)a->out + l0 * a->layer_stride_o;
+    ag.n_layers = nl;
+    st = tr_tree_attention(ctx, &ag, stream);
+    if (st != TR_OK) return st;
+    TR_CUDA_TRY(cudaEventRecord(ctx->ev_attn[g], s));
+    TR_CUDA_TRY(cudaStreamWaitEvent(ctx->io_out, ctx->ev_attn[g], 0));
+    for (int b = 0; b < B; ++b) {
+      const size_t q_off = (static_cast<size_t>(b) * L + l0) * q_layer;
+      TR_CUDA_TRY(cudaMemcpyAsync((__nv_bfloat16*)io->h_out + q_off, (const __nv_bfloat16*)a->out + q_off, nl * q_layer * esz,
+                                  cudaMemcpyDeviceToHost, ctx->io_out));
     }
   }
   const size_t lg_bytes = sizeof(float) * static_cast<size_t>(B) * N * ctx->vocab;
-  TR_CUDA_TRY(cudaMemcpyAsync(io->d_logits_staging, io->h_logits, lg_bytes, cudaMemcpyHostToDevice, s));
-  st = tr_tree_attention(ctx, a, stream);
-  if (st != TR_OK) return st;
+  TR_CUDA_TRY(cudaMemcpyAsync(io->d_logits_staging, io->h_logits, lg_bytes, cudaMemcpyHostToDevice, ctx->io_in));
+  TR_CUDA_TRY(cudaEventRecord(ctx->ev_logits, ctx->io_in));
+  TR_CUDA_TRY(cudaStreamWaitEvent(s, ctx->ev_logits, 0));
   tr_step_out o = *d_out;
   o.d_next_tree = io->d_tree;
   st = tr_verify_update(ctx, io->d_logits_staging, io->d_tree, &o, stream);
   if (st != TR_OK) return st;
   const int W = ctx->depth_max + 1;
-  TR_CUDA_TRY(cudaMemcpyAsync(io->h_out, a->out, q_elems * esz, cudaMemcpyDeviceToHost, s));
   TR_CUDA_TRY(cudaMemcpyAsync(io->h_n_new, o.d_n_new, sizeof(int32_t) * B, cudaMemcpyDeviceToHost, s));
   TR_CUDA_TRY(cudaMemcpyAsync(io->h_out_tokens, o.d_out_tokens, sizeof(int32_t) * B * W, cudaMemcpyDeviceToHost, s));
   TR_CUDA_TRY(cudaMemcpyAsync(io->h_next_tree, io->d_tree, sizeof(int32_t) * B * N, cudaMemcpyDeviceToHost, s));
+  TR_CUDA_TRY(cudaEventRecord(ctx->ev_out, ctx->io_out));
+  TR_CUDA_TRY(cudaStreamWaitEvent(s, ctx->ev_out, 0));  // the caller's stream ends after the last copy out
   TR_CUDA_TRY(cudaStreamSynchronize(s));
   return TR_OK;
 }
