@@ -264,6 +264,49 @@ def test_attention_group_sizes(harness, hq, hkv):
     _attention_case(harness, w, 2, splits=2)
 
 
+@pytest.mark.parametrize("head_dim", [128, 64])
+def test_attention_other_memory_layouts_and_explicit_scale(harness, tr, head_dim):
+    """The same tensors in other layouts - token-major caches [B, L, R, Hkv, D], head-major queries and outputs
+    [B, L, Hq, N, D], a padded last-but-one stride - addressed through the stride arguments, with a scale that is not
+    1/sqrt(head_dim)."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=4, n_kv_heads=2, head_dim=head_dim, ctx=(140, 77))
+    L, scale = 2, 0.11
+    parent, rank = tr.tr_template_from_branching(w.branching, w.n_nodes)
+    ctx = tr.tr_init(w.vocab, w.k, parent, rank, batch=w.batch)
+    q, k, v = synth.attention_inputs(w, L)                              # [B,L,N,Hq,D], [B,L,Hkv,R,D]
+    dq, dk, dv = (harness.bf16_tensor(x, "cuda") for x in (q, k, v))
+    B, N, Hq, Hkv, D = w.batch, w.n_nodes, w.n_q_heads, w.n_kv_heads, head_dim
+    R = k.shape[3]
+    # token-major caches with 8 elements of padding after every (token, head) row group
+    k_tm = torch.zeros(B, L, R, Hkv, D + 8, dtype=torch.bfloat16, device="cuda")
+    v_tm = torch.zeros_like(k_tm)
+    k_tm[..., :D] = dk.permute(0, 1, 3, 2, 4)
+    v_tm[..., :D] = dv.permute(0, 1, 3, 2, 4)
+    k_view, v_view = k_tm[..., :D].permute(0, 1, 3, 2, 4), v_tm[..., :D].permute(0, 1, 3, 2, 4)   # [B,L,Hkv,R,D] views
+    q_hm = dq.permute(0, 1, 3, 2, 4).contiguous()                       # stored [B,L,Hq,N,D]
+    o_hm = torch.zeros_like(q_hm)
+    q_view, o_view = q_hm.permute(0, 1, 3, 2, 4), o_hm.permute(0, 1, 3, 2, 4)
+    d_ctx = torch.tensor(list(w.ctx), dtype=torch.int32, device="cuda")
+    for splits in (0, 2):
+        o_hm.zero_()
+        a = tr.make_attn_args(ctx, q_view, k_view, v_view, o_view, d_ctx, w.max_ctx, scale=scale, splits=splits)
+        tr.tr_tree_attention(ctx, a)
+        torch.cuda.synchronize()
+        got = o_view.float().cpu().numpy()
+        for b in range(B):
+            for l in range(L):
+                c = w.ctx[b]
+                ref = orc.tree_attention(synth.bf16_bits_to_f32(q[b, l]).astype(np.float64),
+                                         synth.bf16_bits_to_f32(k[b, l][:, :c + N]).astype(np.float64),
+                                         synth.bf16_bits_to_f32(v[b, l][:, :c + N]).astype(np.float64), c,
+                                         np.asarray(parent), scale=scale)
+                for h in range(Hq):
+                    mx, rel = attention_close(got[b, l, :, h], ref[:, h])
+                    assert mx <= ATOL and rel <= RTOL, (splits, b, l, h, mx, rel)
+    assert tr.tr_device_flags(ctx) == 0
+    tr.tr_destroy(ctx)
+
+
 def test_largest_tree_128_nodes_attention_and_loop(harness):
     # the maximum template size (ancestor masks are 128-bit; the attention tile has 128 query rows)
     w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], branching=(10, 10), n_nodes=128, n_q_heads=2, n_kv_heads=2,
