@@ -4,8 +4,9 @@
 //   warps 0..3  epilogue: thread r normalises output row r out of TMEM and stores it, off the softmax warps' path
 //   warp 8      TMA producer: Q tile (double-buffered, or single with one more ring slot: kQSingle) and a ring of
 //               32 KB K / V tiles (128 keys x 128 dims, bf16, 128-byte swizzle), one mbarrier per ring slot
-//   warp 9      MMA issuer: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM) and
-//               O += P V (P read from TMEM, V as an MN-major shared-memory operand); owns the TMEM allocation
+//   warp 9      MMA issuer 1: S = Q K^T (tcgen05.mma, both operands in shared memory, accumulator in TMEM); owns
+//               the TMEM allocation
+//   warp 10     MMA issuer 2: O += P V (P read from TMEM, V as an MN-major shared-memory operand)
 //   warps 4..7  softmax: thread r owns query row r (= TMEM lane r): loads its S row, applies the ancestor mask
 //               (a 128-bit mask kept in registers, shifted to the tile), exp2 with a lazily updated reference
 //               maximum, writes P (bf16) over S in TMEM, rescales O in TMEM only when the maximum moved by
@@ -45,8 +46,8 @@ constexpr int NST_MAX = 6;       // ring slots (K and V tiles alternate): 5 besi
                                  // single one (kQSingle: long units, where the Q reload between units is negligible)
 constexpr int TILE_BYTES = BK * HD * 2;       // 32 KB
 constexpr int HALF_BYTES = TILE_BYTES / 2;    // one TMA box: 64 dims x 128 rows
-constexpr int NTHREADS = 384;       // warps 0-3 epilogue, 4-7 softmax, 8 TMA producer, 9 MMA issuer, 10-11 idle
-constexpr int WARP_PRODUCER = 8, WARP_MMA = 9;
+constexpr int NTHREADS = 384;       // warps 0-3 epilogue, 4-7 softmax, 8 TMA producer, 9 QK issuer, 10 PV issuer, 11 idle
+constexpr int WARP_PRODUCER = 8, WARP_MMA = 9, WARP_PV = 10;
 // Registers are re-balanced per warpgroup after start-up (setmaxnreg): 12 warps are launched at 168 each.
 constexpr int REGS_EPILOGUE = 112, REGS_SOFTMAX = 240, REGS_CONTROL = 96;
 
@@ -272,70 +273,76 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     }
     __syncwarp();
   } else if (warp == WARP_MMA) {
-    // =========================== MMA issuer ===========================
+    // =========================== MMA issuer 1: S = Q K^T ===========================
+    // The two products are issued by two threads in different warps (this one and WARP_PV): an issue loop is one
+    // thread's dependent instruction stream (waits, descriptor arithmetic, commits), and a single thread issuing
+    // both left the tensor pipe waiting for it.  One flat stream of tiles over all of this CTA's units; tile g uses
+    // S/P buffer g&1 and ring entries 2g (K) and 2g+1 (V).  This thread runs ahead of the PV issuer as far as the
+    // S/P buffers and the ring allow - also across a unit boundary, so the first scores of the next unit are ready
+    // when the softmax warps finish the current one.
     if (lane == 0) {
       constexpr uint32_t IDESC_QK = make_idesc(false);
-      constexpr uint32_t IDESC_PV = make_idesc(true);
-      // One flat stream of tiles over all of this CTA's units.  Tile g uses S/P buffer g&1 and ring entries 2g (K)
-      // and 2g+1 (V).  The QK of tile g+1 is issued before the PV of tile g - also across a unit boundary, so the
-      // first scores of the next unit are ready when the softmax warps finish the current one.
       bool ok = true;
-      TileCursor kc, vc;
+      TileCursor kc;
       kc.init(p, s_ctx);
-      vc.init(p, s_ctx);
-      auto issue_qk = [&]() -> bool {  // S = Q K^T of the tile under kc
+      while (ok && kc.valid) {
         const uint32_t sb = kc.g & 1u, c = 2u * kc.g, slot = c % NST, qb = kQSingle ? 0u : (kc.ui & 1u);
-        bool w = true;
-        if (kc.j == 0) WAITACC(4, w = mbar_wait(bar(BAR_QFULL + qb), (kQSingle ? kc.ui : (kc.ui >> 1)) & 1u, s_abort))
-        if (!w) return false;
+        if (kc.j == 0) {
+          ok = mbar_wait(bar(BAR_QFULL + qb), (kQSingle ? kc.ui : (kc.ui >> 1)) & 1u, s_abort);
+          if (!ok) break;
+        }
         // the S/P buffer is free once the PV of tile g-2 has completed
-        WAITACC(3, w = mbar_wait(bar(BAR_PVDONE + sb), ((kc.g >> 1) & 1u) ^ 1u, s_abort))
-        if (!w) return false;
-        WAITACC(1, w = mbar_wait(bar(BAR_FULL + slot), (c / NST) & 1u, s_abort))
-        if (!w) return false;
+        ok = mbar_wait(bar(BAR_PVDONE + sb), ((kc.g >> 1) & 1u) ^ 1u, s_abort);
+        if (!ok) break;
+        ok = mbar_wait(bar(BAR_FULL + slot), (c / NST) & 1u, s_abort);
+        if (!ok) break;
         tc_fence_after();
-        const uint32_t qa = base + SM_Q + qb * TILE_BYTES, ka = base + SM_RING + slot * TILE_BYTES;
+        // descriptors are stepped by adding to their low words, to keep the instruction stream short
+        const uint32_t q_lo = smem_desc_lo(base + SM_Q + qb * TILE_BYTES, 16);
+        const uint32_t k_lo = smem_desc_lo(base + SM_RING + slot * TILE_BYTES, 16);
+        const uint32_t s_tm = tmem + sb * 128u;
 #pragma unroll
         for (int k = 0; k < HD / 16; ++k) {
-          const uint32_t off = (k >> 2) * HALF_BYTES + (k & 3) * 32;
-          tc_mma_ss(tmem + sb * 128u, smem_desc(qa + off, 16, 1024), smem_desc(ka + off, 16, 1024), IDESC_QK, k > 0);
+          const uint32_t off16 = static_cast<uint32_t>(((k >> 2) * HALF_BYTES + (k & 3) * 32) >> 4);
+          tc_mma_ss_lh(s_tm, q_lo + off16, k_lo + off16, smem_desc_hi(1024), IDESC_QK, k > 0);
         }
         tc_commit(bar(BAR_EMPTY + slot));                          // K tile consumed
         tc_commit(bar(BAR_SFULL + sb));                            // S ready for the softmax warps
         if (kc.j == kc.nt - 1) tc_commit(bar(BAR_QEMPTY + qb));    // unit's last QK: Q buffer free when it finishes
-        if (kc.j == 0) USTAMP(1, kc.ui, 0)
         kc.next(p, s_ctx);
-        return true;
-      };
-      if (kc.valid) ok = issue_qk();
+      }
+    }
+    __syncwarp();
+  } else if (warp == WARP_PV) {
+    // =========================== MMA issuer 2: O += P V ===========================
+    if (lane == 0) {
+      constexpr uint32_t IDESC_PV = make_idesc(true);
+      bool ok = true;
+      TileCursor vc;
+      vc.init(p, s_ctx);
       while (ok && vc.valid) {
-        if (kc.valid) {
-          ok = issue_qk();
-          if (!ok) break;
-        }
         const uint32_t sb = vc.g & 1u, ob = vc.ui & 1u, c = 2u * vc.g + 1u, vslot = c % NST;
         if (vc.j == 0) {  // the O buffer must have been drained by the epilogue of unit ui-2
           ok = mbar_wait(bar(BAR_OFREE + ob), ((vc.ui >> 1) & 1u) ^ 1u, s_abort);
           if (!ok) break;
         }
-        WAITACC(2, ok = mbar_wait(bar(BAR_PFULL + sb), (vc.g >> 1) & 1u, s_abort))
+        ok = mbar_wait(bar(BAR_FULL + vslot), (c / NST) & 1u, s_abort);
         if (!ok) break;
-        WAITACC(5, ok = mbar_wait(bar(BAR_FULL + vslot), (c / NST) & 1u, s_abort))
+        ok = mbar_wait(bar(BAR_PFULL + sb), (vc.g >> 1) & 1u, s_abort);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t va = base + SM_RING + vslot * TILE_BYTES;
+        const uint32_t v_lo = smem_desc_lo(base + SM_RING + vslot * TILE_BYTES, HALF_BYTES);
+        const uint32_t o_tm = tmem + 256u + ob * 128u, p_tm = tmem + sb * 128u;
+        const uint32_t acc0 = vc.j > 0 ? 1u : 0u;
 #pragma unroll
         for (int k = 0; k < BK / 16; ++k) {
           // A = P (bf16 pairs, 8 TMEM columns per 16 keys); B = V tile, MN-major: 64-dim chunks 16 KB apart,
           // 8-key groups 1 KB apart, 16 keys per step = 2 KB
-          tc_mma_ts(tmem + 256u + ob * 128u, tmem + sb * 128u + k * 8u, smem_desc(va + k * 2048, HALF_BYTES, 1024),
-                    IDESC_PV, (vc.j > 0 || k > 0) ? 1u : 0u);
+          tc_mma_ts_lh(o_tm, p_tm + k * 8u, v_lo + k * (2048u >> 4), smem_desc_hi(1024), IDESC_PV, k > 0 ? 1u : acc0);
         }
         tc_commit(bar(BAR_EMPTY + vslot));                             // V tile consumed
         tc_commit(bar(BAR_PVDONE + sb));                               // P consumed, O updated
         if (vc.j == vc.nt - 1) tc_commit(bar(BAR_OREADY + ob));        // the unit's output is complete
-        if (vc.j == 0) USTAMP(1, vc.ui, 1)
-        if (vc.j == vc.nt - 1) USTAMP(1, vc.ui, 2)
         vc.next(p, s_ctx);
       }
     }
