@@ -369,9 +369,9 @@ def run_ours(args, w):
 
 # DRAM bytes (read + write) of one attention launch from the committed ncu capture (see profiles/), per workload.
 NCU_TRAFFIC_BYTES = {
-    # profiles/tr_attn_tc_kernel_llama2-7b_16layers.md: (300.13 MB read + 5.04 MB written) per 16-layer launch,
+    # profiles/tr_attn_tc_kernel_llama2-7b_16layers.md: (300.03 MB read + 4.92 MB written) per 16-layer launch,
     # scaled to the 32 layers of one benchmark launch (traffic is proportional to the layers processed)
-    "llama2-7b": 2 * (300_127_488 + 5_039_872),
+    "llama2-7b": 2 * (300_028_928 + 4_923_136),
 }
 
 
