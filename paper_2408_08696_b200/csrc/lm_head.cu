@@ -193,20 +193,23 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           const int v = cbase + c0 + i;
-          float cv = __uint_as_float(x[i]);
+          const float cv = __uint_as_float(x[i]);
           // ascending vocabulary order + strict comparisons: among equal values the lower index stays in front
           if (v < vlim && cv > val[KMAX - 1]) {
-            int ci = v;
+            // Insert into the sorted list without a serial chain: entry t keeps its value if the new one does not
+            // beat it, takes its upper neighbour's if the new one beats that too, and the new one otherwise.  Every
+            // entry depends on two comparisons only (a compare-and-swap cascade costs ~8 dependent steps, and the
+            // 32 rows of a warp insert at different columns, so nearly every column pays one insertion per warp).
+            bool gt[KMAX];
 #pragma unroll
-            for (int t = 0; t < KMAX; ++t) {
-              const bool sw = cv > val[t];
-              const float tv = val[t];
-              const int ti = idx[t];
-              val[t] = sw ? cv : tv;
-              idx[t] = sw ? ci : ti;
-              cv = sw ? tv : cv;
-              ci = sw ? ti : ci;
+            for (int t = 0; t < KMAX; ++t) gt[t] = cv > val[t];
+#pragma unroll
+            for (int t = KMAX - 1; t > 0; --t) {
+              val[t] = gt[t] ? (gt[t - 1] ? val[t - 1] : cv) : val[t];
+              idx[t] = gt[t] ? (gt[t - 1] ? idx[t - 1] : v) : idx[t];
             }
+            val[0] = gt[0] ? cv : val[0];
+            idx[0] = gt[0] ? v : idx[0];
           }
         }
       }
