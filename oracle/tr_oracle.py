@@ -295,6 +295,48 @@ def verify_update(M, S, logits, parent, rank, rule="last", only_accepted=False):
 
 
 # --------------------------------------------------------------------------
+# Verification under temperature sampling (Sec. 5.3 "Temperature Sampling").
+# The paper reports that TR keeps working at temperatures 0.3 - 1.0 and explains
+# the slight loss by sampled tokens falling outside the stored top-k; it does not
+# spell the acceptance rule out.  Reading used here ("sample, then match"): every
+# node draws ONE token from its output distribution at temperature T, and a draft
+# child is correct iff it equals the token drawn at its parent - greedy
+# verification with the argmax replaced by the draw, which emits exactly the
+# tokens that token-by-token sampling with the same draws would.  The draw is
+# written as a Gumbel-max so that it is an argmax of per-element float32
+# arithmetic (no summation order): x = argmax_v ( logits[v] / T + g[v] ),
+# g = -log(-log(u)), u uniform; the noise g is an INPUT (the caller's generator).
+# --------------------------------------------------------------------------
+def sample_tokens(logits, gumbel, inv_temperature):
+    """Token drawn at every node: argmax_v of z[v] = fl32(fl32(logits[v] * inv_temperature) + gumbel[v]), lowest
+    index among equal z (float32 multiply, then float32 add: two roundings, the decision precision of the kernel).
+    With gumbel == 0 this is the greedy argmax for any inv_temperature > 0.
+    Pinned by: gumbel = 0 gives argtopk's column 0; empirical frequencies of many draws against softmax(logits / T)
+    (the Gumbel-max theorem); a hand case where the noise overturns the argmax.
+    """
+    logits = np.asarray(logits, dtype=np.float32)
+    gumbel = np.asarray(gumbel, dtype=np.float32)
+    z = (logits * np.float32(inv_temperature)).astype(np.float32) + gumbel
+    return argtopk(z.astype(np.float32), 1)[:, 0]
+
+
+def verify_update_sampled(M, S, logits, gumbel, inv_temperature, parent, rank, rule="last", only_accepted=False):
+    """verify_update with the draw of sample_tokens in place of the argmax for acceptance and for the extra token;
+    the matrix still stores argtopk(logits) of every node (the candidates are the model's top-k, whatever was
+    drawn - which is why, in the paper's words, draws outside the top-k cost acceptance at high temperature).
+    M is modified in place.  Returns verify_update's dict plus `sampled`.
+    """
+    k = M.shape[1]
+    O = argtopk(logits, k)
+    x = sample_tokens(logits, gumbel, inv_temperature)
+    n_new, acc_nodes, out_tokens, next_root = accept(S, x, parent)
+    update_matrix(M, S, O, rule=rule, nodes=acc_nodes if only_accepted else None)
+    nxt = bfs_tree(M, parent, rank, next_root)
+    return dict(topk=O, sampled=x, n_new=n_new, acc_nodes=acc_nodes, out_tokens=out_tokens,
+                next_root=next_root, next_tree=nxt)
+
+
+# --------------------------------------------------------------------------
 # Commit of the accepted path (Sec. 5.4: "updating the matrix, input tokens, and key-value cache")
 # --------------------------------------------------------------------------
 def commit(k, v, ctx_len, tokens, acc_nodes, out_tokens):

@@ -102,7 +102,7 @@ def pool_slice(pool, off, shape):
 
 
 STREAM_Q, STREAM_K, STREAM_V, STREAM_NOISE, STREAM_SUCC, STREAM_M, STREAM_ROOT = 10, 11, 12, 13, 14, 15, 16
-STREAM_HID, STREAM_W = 17, 18
+STREAM_HID, STREAM_W, STREAM_GUMBEL = 17, 18, 19
 
 
 def attention_inputs(w: Workload, n_layers=None, pool=None):
@@ -169,6 +169,14 @@ def noise_logits(w: Workload, n_rot=4):
     """float32 [n_rot, B, N, V] N(0,1) noise matrices that rotate over steps."""
     return _rng(w.seed, STREAM_NOISE).standard_normal(
         (n_rot, w.batch, w.n_nodes, w.vocab), dtype=np.float32)
+
+
+def gumbel_noise(w: Workload, n_rot=4):
+    """float32 [n_rot, B, N, V] standard Gumbel draws g = -log(-log(u)), u uniform in (0, 1): the random numbers of
+    temperature sampling, rotating over steps like the noise logits."""
+    u = _rng(w.seed, STREAM_GUMBEL).random((n_rot, w.batch, w.n_nodes, w.vocab), dtype=np.float32)
+    u = np.clip(u, np.float32(1e-20), np.float32(1.0 - 2.0 ** -24))
+    return (-np.log(-np.log(u.astype(np.float64)))).astype(np.float32)
 
 
 def zipf_successors(w: Workload):

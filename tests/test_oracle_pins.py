@@ -454,3 +454,66 @@ def test_lm_head_synthetic_inputs():
     # small-integer inputs: the logits are exact integers, identical in float32 and float64
     _, logits = orc.lm_head_topk(fi, fw, w.k)
     assert np.array_equal(logits, np.round(logits)) and np.array_equal(logits.astype(np.float32).astype(np.float64), logits)
+
+
+# ---------------------------------------------------------------------------
+# Temperature sampling (Sec. 5.3): the draw as a Gumbel-max, then greedy-style matching
+# ---------------------------------------------------------------------------
+def test_sample_tokens_without_noise_is_the_argmax_and_noise_can_overturn_it():
+    r = np.random.default_rng(11)
+    logits = r.standard_normal((9, 40)).astype(np.float32)
+    logits[3, 7] = logits[3, 21] = logits[3].max() + 1      # a tie: the lower index wins
+    zero = np.zeros_like(logits)
+    for inv_t in (1.0, 0.25, 3.0):
+        assert np.array_equal(orc.sample_tokens(logits, zero, inv_t), orc.argtopk(logits, 1)[:, 0])
+    # hand case: logits (2, 1, 0) at T = 0.5 -> scaled (4, 2, 0); noise (0, 3, 0) makes index 1 the draw (5 > 4)
+    lg = np.array([[2.0, 1.0, 0.0]], dtype=np.float32)
+    assert orc.sample_tokens(lg, np.array([[0.0, 3.0, 0.0]], dtype=np.float32), 2.0)[0] == 1
+    assert orc.sample_tokens(lg, np.array([[0.0, 1.5, 0.0]], dtype=np.float32), 2.0)[0] == 0
+
+
+def test_sample_tokens_follow_the_softmax_at_temperature():
+    """Gumbel-max theorem: the frequencies of many draws match softmax(logits / T)."""
+    r = np.random.default_rng(12)
+    logits = np.array([1.5, 0.3, -0.2, 2.0, 0.0, -1.0], dtype=np.float32)
+    for T in (0.5, 1.0):
+        n = 60000
+        u = r.random((n, logits.size))
+        g = (-np.log(-np.log(u))).astype(np.float32)
+        draws = orc.sample_tokens(np.broadcast_to(logits, (n, logits.size)), g, 1.0 / T)
+        freq = np.bincount(draws, minlength=logits.size) / n
+        p = np.exp(logits.astype(np.float64) / T)
+        p /= p.sum()
+        assert np.abs(freq - p).max() < 4 * np.sqrt(0.25 / n) + 1e-3      # four standard errors of a proportion
+
+
+def test_sampled_verification_equals_token_by_token_sampling():
+    """Losslessness under sampling: TR with 'sample, then match' emits exactly the tokens that token-by-token
+    decoding with the same per-position draws emits (toy model: logits depend on the last token only, the draw at a
+    position uses that position's noise row)."""
+    r = np.random.default_rng(13)
+    V, k, steps = 50, 4, 20
+    parent, rank = orc.template_from_branching((3, 2, 1), 12)
+    table = r.standard_normal((V, V)).astype(np.float32) * 2      # next-token logits given the last token
+    M = r.integers(0, V, size=(V, k)).astype(np.int64)
+    root = 5
+    # one noise row per absolute position, so both decoders see the same randomness
+    noise = (-np.log(-np.log(r.random((400, V))))).astype(np.float32)
+    inv_t = 1.0 / 0.7
+    # token-by-token
+    ref = [root]
+    for pos in range(300):
+        ref.append(int(orc.sample_tokens(table[ref[-1]][None], noise[pos][None], inv_t)[0]))
+    # TR: node i of the tree sits at position pos + depth(i); its draw uses that position's noise row
+    depth = orc.node_depth(parent)
+    out = [root]
+    S = orc.bfs_tree(M, parent, rank, root)
+    for _ in range(steps):
+        pos = len(out) - 1
+        logits = table[S]                                          # [N, V]
+        g = noise[pos + np.asarray(depth)]
+        rec = orc.verify_update_sampled(M, S, logits, g, inv_t, parent, rank)
+        out.extend(rec["out_tokens"])
+        S = rec["next_tree"]
+    assert out == ref[:len(out)]
+    assert len(out) - 1 > steps        # some drafts were accepted
