@@ -194,6 +194,52 @@ def measure_lm_head(torch, tr, dw, w, dev, reps=20):
             "device_flags": tr.tr_device_flags(dw.ctx)}
 
 
+def measure_sampled_verify(torch, tr, dw, w, dev, reps=20):
+    """Verification under temperature sampling on the step's logits (not part of the timed step, which is greedy):
+    tr_verify_update_sampled as a CUDA graph replayed `reps` times on its own copy of the loop state, beside the
+    greedy tr_verify_update timed the same way.  Two passes over the logits and one over the noise."""
+    from paper_2408_08696_b200 import synth
+    rows = w.batch * w.n_nodes
+    gen = torch.Generator(device=dev).manual_seed((w.seed + 7) & 0x7FFFFFFF)
+    u = torch.rand(w.batch, w.n_nodes, w.vocab, device=dev, generator=gen).clamp_(1e-20, 1.0 - 2.0 ** -24)
+    d_g = -torch.log(-torch.log(u))
+    d_tree = dw.d_tree.clone()
+    out_struct, out = tr.make_step_out(dw.ctx)
+    out_struct.d_next_tree = d_tree.data_ptr()
+    M0 = [tr.tr_matrix_export(dw.ctx, b) for b in range(w.batch)]      # the measurement must not disturb the loop
+    res = {}
+    for name in ("sampled", "greedy"):
+        s = torch.cuda.Stream(dev)
+        graph = torch.cuda.CUDAGraph()
+
+        def call(stream=None):
+            if name == "sampled":
+                tr.tr_verify_update_sampled(dw.ctx, dw.d_logits[0], d_g, 1.0 / 0.7, d_tree, out_struct, stream=stream)
+            else:
+                tr.tr_verify_update(dw.ctx, dw.d_logits[0], d_tree, out_struct, stream)
+        call()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(graph, stream=s):
+                call(s)
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            graph.replay()
+        e1.record()
+        torch.cuda.synchronize()
+        res[name] = e0.elapsed_time(e1) / reps * 1000.0
+    for b in range(w.batch):
+        tr.tr_matrix_import(dw.ctx, b, M0[b])
+    byts = rows * w.vocab * 4 * 3
+    return {"us": res["sampled"], "greedy_verify_update_us": res["greedy"], "algorithmic_bytes": byts,
+            "achieved": byts / res["sampled"] / 1e3, "unit": "GB/s", "temperature": 0.7, "gpu_launches": 3,
+            "device_flags": tr.tr_device_flags(dw.ctx)}
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -325,6 +371,7 @@ def run_ours(args, w):
     e2e = replicas.aggregate(e2e_ms, Ke, device=dev if world > 1 else "cpu")
 
     lm = measure_lm_head(torch, tr, dw, w, dev) if rank == 0 else None
+    sampled_verify = measure_sampled_verify(torch, tr, dw, w, dev) if rank == 0 else None
 
     if rank == 0:
         peak, peak_src = load_peaks()
@@ -358,7 +405,8 @@ def run_ours(args, w):
             "gpu_launches": dw.kernels_per_step() * K,
             "clocks": clocks,
             "mean_new_tokens_per_step": n_new_sum / (B * n_stat),
-            "next_rows": {"lm_head_topk": dict(lm, frac=lm["achieved"] / peak, peak=peak)},
+            "next_rows": {"lm_head_topk": dict(lm, frac=lm["achieved"] / peak, peak=peak),
+                          "verify_update_sampled": sampled_verify},
             "device_flags": flags,
         }
         print(json.dumps(line), flush=True)

@@ -155,6 +155,25 @@ int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appe
 tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream);
 
 /*
+ * Verification under temperature sampling (Sec. 5.3 "Temperature Sampling": TR keeps its speed-up at T = 0.3 .. 1.0 and
+ * loses a little when drawn tokens fall outside the stored top-k; the paper does not spell the acceptance rule out).
+ * Rule implemented ("sample, then match"): every node i draws one token
+ *     x_i = argmax_v ( fl32( fl32(logits[i,v] * inv_temperature) + gumbel[i,v] ) ),   lowest v among equal values,
+ * which for standard Gumbel noise g = -log(-log(u)) is a draw from softmax(logits[i] / T), T = 1 / inv_temperature
+ * (Gumbel-max); a draft child c is correct iff tree[c] == x_parent(c); out_tokens are the accepted drafts followed by
+ * the draw of the last accepted node.  Everything else is tr_verify_update: M_b[tree[i]] = argtopk(logits[i]) for
+ * every node (the stored candidates are the model's top-k, not the draws), next tree from the updated matrix.
+ * The emitted tokens are exactly those of token-by-token sampling with the same noise.  With gumbel == 0 the call
+ * equals tr_verify_update.
+ * DEVICE in : d_logits, d_gumbel [batch, N, V] fp32 (the noise is the caller's: any generator, one row per node);
+ *             inv_temperature > 0 and finite (else TR_ERR_INVALID_ARG); d_tree [batch, N].
+ * DEVICE out: as tr_verify_update; d_sampled [batch, N] int32 receives the draws (NULL: kept in the context).
+ * Two passes over the logits and one over the noise; allocates nothing, does not synchronise.
+ */
+tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits, const float* d_gumbel, float inv_temperature,
+                                   const int32_t* d_tree, const tr_step_out* out, int32_t* d_sampled, void* stream);
+
+/*
  * Output layer fused with argtopk (Sec. 2.1: p = M(x), x^0..x^{k-1} = argtopk(p); Sec. 5.4: the forward pass is most of
  * a step).  For the rows = batch * N tree nodes,
  *     logits[r, v] = sum_h hidden[r, h] * weight[v, h]      bf16 inputs, fp32 accumulation on the tensor cores

@@ -92,6 +92,8 @@ lib.tr_commit.argtypes = [C.c_void_p, C.POINTER(tr_commit_args), C.c_void_p, C.c
 lib.tr_topk_noalloc.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p]
 lib.tr_topk_noalloc_limits.argtypes = [_P32, _P32]
 lib.tr_verify_update_topk.argtypes = [C.c_void_p, C.c_void_p, C.POINTER(tr_step_out), C.c_void_p]
+lib.tr_verify_update_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_float, C.c_void_p,
+                                         C.POINTER(tr_step_out), C.c_void_p, C.c_void_p]
 lib.tr_lm_head_topk.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p,
                                 C.c_void_p, C.c_void_p]
 lib_synth.trs_patch_logits.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float,
@@ -244,6 +246,24 @@ def tr_verify_update(ctx, d_logits, d_tree, out_struct, stream=None):
     _check(lib.tr_verify_update(ctx.handle, _dev(d_logits, torch.float32, "d_logits"),
                                 _dev(d_tree, torch.int32, "d_tree"), C.byref(out_struct), _stream(stream)),
            "tr_verify_update")
+
+
+def tr_verify_update_sampled(ctx, d_logits, d_gumbel, inv_temperature, d_tree, out_struct, d_sampled=None,
+                             stream=None):
+    """Verification under temperature sampling: d_gumbel is standard Gumbel noise of the logits' shape."""
+    shape = (ctx.batch, ctx.n_nodes, ctx.vocab)
+    if tuple(d_logits.shape) != shape or tuple(d_gumbel.shape) != shape or not d_logits.is_contiguous() \
+            or not d_gumbel.is_contiguous():
+        raise ValueError("d_logits and d_gumbel must be contiguous [batch, N, V]")
+    smp = None
+    if d_sampled is not None:
+        if d_sampled.numel() != ctx.batch * ctx.n_nodes or not d_sampled.is_contiguous():
+            raise ValueError("d_sampled must be contiguous with batch*N elements")
+        smp = _dev(d_sampled, torch.int32, "d_sampled")
+    _check(lib.tr_verify_update_sampled(ctx.handle, _dev(d_logits, torch.float32, "d_logits"),
+                                        _dev(d_gumbel, torch.float32, "d_gumbel"), float(inv_temperature),
+                                        _dev(d_tree, torch.int32, "d_tree"), C.byref(out_struct), smp,
+                                        _stream(stream)), "tr_verify_update_sampled")
 
 
 def tr_verify_update_topk(ctx, d_tree, out_struct, stream=None):

@@ -73,9 +73,10 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
                const int32_t* __restrict__ level_off, int depth_max, const int32_t* tree_in,
                const int32_t* __restrict__ topk_idx, int32_t* __restrict__ n_new, int32_t* __restrict__ acc_nodes,
                int32_t* __restrict__ out_tokens, int32_t* __restrict__ next_root, int32_t* tree_out,
-               uint32_t* __restrict__ flags, const uint32_t* __restrict__ anc, int update_rule, int update_scope) {
+               uint32_t* __restrict__ flags, const uint32_t* __restrict__ anc, int update_rule, int update_scope,
+               const int32_t* __restrict__ target) {
   __shared__ int32_t s_S[TR_MAX_NODES];
-  __shared__ int32_t s_argmax[TR_MAX_NODES];
+  __shared__ int32_t s_argmax[TR_MAX_NODES];  // the token each node's children must match: argmax, or the given draw
   __shared__ int32_t s_tree[TR_MAX_NODES];
   __shared__ uint32_t s_best[TAIL_THREADS / 32];
   __shared__ TailTables tb;
@@ -98,7 +99,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     s_S[tid] = tok;
 #pragma unroll
     for (int c = 0; c < TR_MAX_K; ++c) row[c] = c < k ? topk[tid * k + c] : 0;  // fetched once, with the tokens
-    s_argmax[tid] = row[0];
+    s_argmax[tid] = target ? target[static_cast<size_t>(b) * n + tid] : row[0];
   }
   __syncthreads();
 
@@ -178,11 +179,12 @@ tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tr
   return TR_OK;
 }
 
-tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s) {
+tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s,
+                         const int32_t* d_target) {
   TR_CUDA_TRY(tr_launch_pdl(tr_tail_kernel, dim3(ctx->batch), dim3(TAIL_THREADS), 0, s, ctx->d_M, ctx->vocab, ctx->k,
                             ctx->n_nodes, ctx->d_parent, ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
                             d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes, out->d_out_tokens,
                             out->d_next_root, out->d_next_tree, ctx->d_flags, ctx->d_anc, ctx->update_rule,
-                            ctx->update_scope));
+                            ctx->update_scope, d_target));
   return TR_OK;
 }

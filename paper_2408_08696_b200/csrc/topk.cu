@@ -29,10 +29,14 @@ __device__ __forceinline__ u64 warp_max_u64(u64 x) {
   return (static_cast<u64>(mh) << 32) | ml;
 }
 
-template <bool kVec>
+// kSample: rank z = fl32(fl32(logit * inv_t) + gumbel) instead of the logits (Sec. 5.3 temperature sampling: with k = 1
+// the result is the token drawn at temperature 1 / inv_t by the Gumbel-max rule).  Two roundings, no fused multiply-add:
+// the decision is reproducible with plain float32 arithmetic.
+template <bool kVec, bool kSample = false>
 __global__ void __launch_bounds__(TOPK_THREADS, 5)
 tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __restrict__ part,
-               unsigned int* __restrict__ ticket, int32_t* __restrict__ topk_idx) {
+               unsigned int* __restrict__ ticket, int32_t* __restrict__ topk_idx,
+               const float* __restrict__ gumbel = nullptr, float inv_t = 1.f) {
   constexpr int E = TOPK_ELEMS_PER_THREAD;
   constexpr int G = TOPK_THREADS / 16;  // half-warp groups: 16 >= TR_MAX_K
   __shared__ u64 s_gmax[G];
@@ -61,6 +65,11 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
       idx0[j] = i0;
       float4 t = (i0 < V) ? __ldcs(reinterpret_cast<const float4*>(rowp + i0))
                           : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+      if (kSample && i0 < V) {
+        const float4 g = __ldcs(reinterpret_cast<const float4*>(gumbel + static_cast<size_t>(row) * V + i0));
+        t.x = __fadd_rn(__fmul_rn(t.x, inv_t), g.x); t.y = __fadd_rn(__fmul_rn(t.y, inv_t), g.y);
+        t.z = __fadd_rn(__fmul_rn(t.z, inv_t), g.z); t.w = __fadd_rn(__fmul_rn(t.w, inv_t), g.w);
+      }
       v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
     }
   } else {
@@ -68,6 +77,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
     for (int j = 0; j < E; ++j) {
       const int i = seg_base + j * TOPK_THREADS + tid;
       v[j] = (i < V) ? __ldcs(rowp + i) : -INFINITY;
+      if (kSample && i < V) v[j] = __fadd_rn(__fmul_rn(v[j], inv_t), __ldcs(gumbel + static_cast<size_t>(row) * V + i));
     }
   }
   auto index_of = [&](int j) -> int {
@@ -209,16 +219,31 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __
   }
 }
 
-tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s) {
+tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
+                         const float* d_gumbel, float inv_temperature, int k_override) {
   const int rows = ctx->batch * ctx->n_nodes;
+  const int k = k_override > 0 ? k_override : ctx->k;
   dim3 grid(ctx->topk_segs, rows);
-  const bool vec = (ctx->vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
+  bool vec = (ctx->vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
+  if (d_gumbel) {
+    vec = vec && ((reinterpret_cast<uintptr_t>(d_gumbel) & 15) == 0);
+    if (vec)
+      TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true, true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
+                                ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, d_gumbel,
+                                inv_temperature));
+    else
+      TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false, true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
+                                ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, d_gumbel,
+                                inv_temperature));
+    return TR_OK;
+  }
+  const float* no_noise = nullptr;
   if (vec)
-    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, ctx->k,
-                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx));
+    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true, false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
+                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, no_noise, 1.f));
   else
-    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, ctx->k,
-                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx));
+    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false, false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
+                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, no_noise, 1.f));
   return TR_OK;
 }
 
@@ -282,9 +307,9 @@ extern "C" tr_status tr_topk_noalloc(const float* d_logits, int32_t rows, int32_
   const dim3 grid(segs, rows);
   const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
   if (vec)
-    tr_topk_kernel<true><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx);
+    tr_topk_kernel<true, false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx, nullptr, 1.f);
   else
-    tr_topk_kernel<false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx);
+    tr_topk_kernel<false, false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx, nullptr, 1.f);
   TR_CUDA_TRY(cudaGetLastError());
   return TR_OK;
 }

@@ -62,6 +62,7 @@ static tr_status free_all(tr_ctx* c) {
   cudaFree(c->d_topk_ticket);
   cudaFree(c->d_seq_ticket);
   cudaFree(c->d_lm_part);
+  cudaFree(c->d_sampled);
   if (c->io_in) cudaStreamDestroy(c->io_in);
   if (c->io_out) cudaStreamDestroy(c->io_out);
   for (cudaEvent_t e : {c->ev_start, c->ev_logits, c->ev_out}) if (e) cudaEventDestroy(e);
@@ -149,6 +150,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaMemset(c->d_topk_ticket, 0, sizeof(unsigned int) * rows));
   TR_INIT_TRY(cudaMalloc(&c->d_seq_ticket, sizeof(unsigned int) * batch));
   TR_INIT_TRY(cudaMemset(c->d_seq_ticket, 0, sizeof(unsigned int) * batch));
+  TR_INIT_TRY(cudaMalloc(&c->d_sampled, sizeof(int32_t) * rows));
   c->lm_parts_cap = 2 * c->sm_count;  // two lists per CTA
   TR_INIT_TRY(cudaMalloc(&c->d_lm_part, sizeof(unsigned long long) * rows * c->lm_parts_cap * k));
 
@@ -253,6 +255,26 @@ extern "C" tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const 
   tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s);
   if (st != TR_OK) return st;
   return tr_launch_tail(ctx, d_tree, out, s);
+}
+
+extern "C" tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits, const float* d_gumbel,
+                                              float inv_temperature, const int32_t* d_tree, const tr_step_out* out,
+                                              int32_t* d_sampled, void* stream) {
+  if (!ctx || !d_logits || !d_gumbel || !d_tree || !out) return TR_ERR_INVALID_ARG;
+  if (!(inv_temperature > 0.f) || !(inv_temperature < INFINITY)) return TR_ERR_INVALID_ARG;
+  if (!out->d_topk_idx || !out->d_n_new || !out->d_acc_nodes || !out->d_out_tokens || !out->d_next_root ||
+      !out->d_next_tree)
+    return TR_ERR_INVALID_ARG;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  int32_t* drawn = d_sampled ? d_sampled : ctx->d_sampled;
+  // the candidates stored in the matrix are the model's top-k, whatever is drawn
+  tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s);
+  if (st != TR_OK) return st;
+  // the draw: the first entry of the same ranking applied to logit / T + noise (the scratch lists are reused: the
+  // kernels are ordered on the stream)
+  st = tr_launch_topk(ctx, d_logits, drawn, s, d_gumbel, inv_temperature, 1);
+  if (st != TR_OK) return st;
+  return tr_launch_tail(ctx, d_tree, out, s, drawn);
 }
 
 extern "C" tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream) {

@@ -49,6 +49,7 @@ struct tr_ctx {
   unsigned int* d_topk_ticket = nullptr;      // [batch*N]
   unsigned int* d_seq_ticket = nullptr;       // [batch]: CTAs of a sequence that passed tr_commit's read phase
   int topk_segs = 0;
+  int32_t* d_sampled = nullptr;               // [batch*N] tokens drawn by tr_verify_update_sampled
   unsigned long long* d_lm_part = nullptr;    // [batch*N][lm_parts_cap][k] per-CTA lists of tr_lm_head_topk
   int lm_parts_cap = 0;
   float* d_attn_part_o = nullptr;   // [slots][128][128]
@@ -84,8 +85,13 @@ __device__ __forceinline__ void tr_grid_dependency_wait() { asm volatile("gridde
 #endif
 
 // launchers (host functions defined next to their kernels)
-tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s);
-tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s);
+// With d_gumbel: the kernel ranks z = fl32(fl32(logit * inv_temperature) + gumbel) instead of the logits, k_override
+// entries per row (1: the draw of temperature sampling).
+tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
+                         const float* d_gumbel = nullptr, float inv_temperature = 1.f, int k_override = 0);
+// d_target [batch, N] (optional): the token every node's children are matched against, instead of topk[:, 0]
+tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s,
+                         const int32_t* d_target = nullptr);
 tr_status tr_launch_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,
                            const int32_t* d_out_tokens, const int32_t* d_n_new, cudaStream_t s);
 tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);
