@@ -19,25 +19,6 @@
 #include "tc_ptx.cuh"
 #include "tr_internal.cuh"
 
-// Optional timeline instrumentation (off in normal builds): with -DTR_TC_STAMPS=<cta+1> the chosen CTA records
-// SM-clock stamps of a few events per unit, read back with tr_debug_stamps().
-#ifndef TR_TC_STAMPS
-#define TR_TC_STAMPS 0
-#endif
-#if TR_TC_STAMPS
-__device__ long long g_stamps[4 * 16 * 8];
-#define WAITACC(k, expr) { const long long w0__ = clock64(); expr; if (blockIdx.x == TR_TC_STAMPS - 1) g_stamps[(0 * 16 + 15) * 8 + (k)] += clock64() - w0__; }
-#define USTAMP(role, unit, k) \
-  { if (blockIdx.x == TR_TC_STAMPS - 1 && (unit) < 16) g_stamps[((role) * 16 + (unit)) * 8 + (k)] = clock64(); }
-extern "C" int tr_debug_stamps(long long* host) {
-  cudaDeviceSynchronize();
-  return static_cast<int>(cudaMemcpyFromSymbol(host, g_stamps, sizeof(long long) * 4 * 16 * 8));
-}
-#else
-#define USTAMP(role, unit, k) {}
-#define WAITACC(k, expr) { expr; }
-#endif
-
 namespace {
 
 constexpr int BK = 128;          // keys per tile
@@ -245,7 +226,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const Unit x = decode_unit(p, u, s_ctx);
         if (x.t0 >= x.t1) continue;
         const uint32_t qb = kQSingle ? 0u : (ui & 1u);
-        USTAMP(0, ui, 0)
         ok = mbar_wait(bar(BAR_QEMPTY + qb), ((kQSingle ? ui : (ui >> 1)) & 1u) ^ 1u, s_abort);
         if (!ok) break;
         mbar_expect_tx(bar(BAR_QFULL + qb), TILE_BYTES);
@@ -256,7 +236,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
             const uint32_t slot = c % NST, par = ((c / NST) & 1u) ^ 1u;
-            WAITACC(0, ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort))
+            ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort);
             if (!ok) break;
             const CUtensorMap* m = kv == 0 ? &map_k : &map_v;
             const uint32_t dst = base + SM_RING + slot * TILE_BYTES;
@@ -265,9 +245,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tma_load_5d_hint(dst + HALF_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b, pol);
             ++c;
           }
-          if (t == x.t0) USTAMP(0, ui, 1)
         }
-        USTAMP(0, ui, 2)
         ++ui;
       }
     }
@@ -372,7 +350,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
         if (!ok) break;
         tc_fence_after();
-        if (tid == 128 && j == 0) USTAMP(2, ui, 0)
         uint32_t sreg[4][32];
 #pragma unroll
         for (int q = 0; q < 4; ++q) tc_ld32(tmem + lane_base + sb * 128u + q * 32u, sreg[q]);
@@ -472,8 +449,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         tc_wait_st();
         tc_fence_before();
         mbar_arrive(bar(BAR_PFULL + sb));
-        if (tid == 128 && j == 0) USTAMP(2, ui, 1)
-        if (tid == 128 && j == nt - 1) USTAMP(2, ui, 2)
       }
       if (!ok) break;
       if (nt <= 0) continue;  // empty split: the epilogue warps write its (empty) partial
@@ -485,7 +460,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       s_lm[ob * 256 + r] = l;
       s_lm[ob * 256 + 128 + r] = m_ref;
       mbar_arrive(bar(BAR_LFULL + ob));
-      if (tid == 128) USTAMP(2, ui, 3)
       ++ui;
     }
   } else {
@@ -518,7 +492,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
-      if (tid == 0) USTAMP(3, ui, 0)
       const float l = s_lm[ob * 256 + r], m_ref = s_lm[ob * 256 + 128 + r];
       const float inv = 1.f / l;
       __nv_bfloat16* orow = p.out + x.b * p.os_b + x.layer * p.os_l + head * p.os_h + static_cast<int64_t>(node) * p.os_t;
@@ -557,7 +530,6 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         pml[0] = m_ref;
         pml[1] = l;
       }
-      if (tid == 0) USTAMP(3, ui, 1)
       ++ui;
     }
   }
