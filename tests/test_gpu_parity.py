@@ -463,20 +463,23 @@ def test_decode_loop_with_commit_grows_the_prefix(tr):
 
 
 # ------------------------------------------------------------------ whole step, host-buffer entry point
-def test_step_host_matches_device_calls(harness, tr):
-    import ctypes as C
-    w = dataclasses.replace(synth.WORKLOADS["tiny"], ctx=(100,))
-    L = 2
+@pytest.mark.parametrize("ctxs,L", [((100,), 2), ((100, 37, 64), 5)])
+def test_step_host_matches_device_calls(harness, tr, ctxs, L):
+    """The host-buffer entry point (copies pipelined over two layer groups, one strided copy per sequence and group
+    for the tree K/V rows): one sequence, and three sequences with different prefix lengths over five layers."""
+    w = dataclasses.replace(synth.WORKLOADS["tiny"], ctx=ctxs)
     dw = harness.DeviceWorkload(w, n_layers=L)
     ol = OracleLoop(w)
     B, N, V, Hq, Hkv, D = w.batch, w.n_nodes, w.vocab, w.n_q_heads, w.n_kv_heads, w.head_dim
     q, k, v = synth.attention_inputs(w, L)
-    c = w.ctx[0]
     h_q = torch.from_numpy(q.view(np.int16)).pin_memory()
-    h_tk = torch.from_numpy(np.ascontiguousarray(k[:, :, :, c:c + N]).view(np.int16)).pin_memory()
-    h_tv = torch.from_numpy(np.ascontiguousarray(v[:, :, :, c:c + N]).view(np.int16)).pin_memory()
-    dw.k[:, :, :, c:c + N] = 0          # the call itself must place the tree rows
-    dw.v[:, :, :, c:c + N] = 0
+    tk = np.stack([k[b, :, :, c:c + N] for b, c in enumerate(w.ctx)])
+    tv = np.stack([v[b, :, :, c:c + N] for b, c in enumerate(w.ctx)])
+    h_tk = torch.from_numpy(np.ascontiguousarray(tk).view(np.int16)).pin_memory()
+    h_tv = torch.from_numpy(np.ascontiguousarray(tv).view(np.int16)).pin_memory()
+    for b, c in enumerate(w.ctx):       # the call itself must place the tree rows
+        dw.k[b, :, :, c:c + N] = 0
+        dw.v[b, :, :, c:c + N] = 0
     logits = np.stack([synth.step_logits(ol.noise[0, b], ol.S[b], ol.succ, w.boost) for b in range(B)])
     h_logits = torch.from_numpy(logits).pin_memory()
     h_ctx = np.array(w.ctx, dtype=np.int32)
@@ -494,12 +497,14 @@ def test_step_host_matches_device_calls(harness, tr):
     tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)
     recs = ol.step(0)
     compare_step(recs, dw.snapshot(), dw.ctx.max_new)
-    assert h_n_new[0].item() == recs[0]["n_new"]
-    assert h_tokens[0, : recs[0]["n_new"]].tolist() == recs[0]["out_tokens"]
-    assert (h_next[0].numpy() == recs[0]["next_tree"]).all()
-    for l in range(L):
-        ref = oracle_attention(w, q, k, v, 0, l, dw.parent)
-        for h in range(Hq):
-            mx, rel = attention_close(h_out[0, l, :, h].float().numpy(), ref[:, h])
-            assert mx <= ATOL and rel <= RTOL
+    for b in range(B):
+        assert h_n_new[b].item() == recs[b]["n_new"]
+        assert h_tokens[b, : recs[b]["n_new"]].tolist() == recs[b]["out_tokens"]
+        assert (h_next[b].numpy() == recs[b]["next_tree"]).all()
+        for l in range(L):
+            ref = oracle_attention(w, q, k, v, b, l, dw.parent)
+            for h in range(Hq):
+                mx, rel = attention_close(h_out[b, l, :, h].float().numpy(), ref[:, h])
+                assert mx <= ATOL and rel <= RTOL
+    assert tr.tr_device_flags(dw.ctx) == 0
     dw.close()
