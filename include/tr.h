@@ -45,7 +45,7 @@ typedef int32_t tr_status;
 #define TR_MAX_K 16
 
 /* Device flag bits (tr_device_flags). */
-#define TR_FLAG_BAD_TOKEN 1u    /* a tree/root token id was outside [0, V): row skipped / id clamped to 0 */
+#define TR_FLAG_BAD_TOKEN 1u    /* a token id (tree, root, given top-k or draw) was outside [0, V): row skipped / id replaced by 0 */
 #define TR_FLAG_WAIT_TIMEOUT 2u /* a bounded wait inside a kernel ran out (should never happen) */
 #define TR_FLAG_CACHE_FULL 4u   /* tr_commit: no room for another tree behind the grown prefix; sequence left as is */
 
@@ -68,7 +68,7 @@ tr_status tr_template_from_branching(const int32_t* b, int32_t nb, int32_t max_n
  * HOST in: parent[n_nodes], rank[n_nodes] - the static tree in layer order: parent[0] = -1, 0 <= parent[i] < i,
  *   depth non-decreasing, 0 <= rank[i] < k (rank = the column of M a node is drawn from, Appendix tree figure).
  * Errors: TR_ERR_INVALID_ARG (vocab < k, k < 1 or > TR_MAX_K, batch < 1, NULL), TR_ERR_TEMPLATE
- *   (malformed tree, n_nodes > TR_MAX_NODES), TR_ERR_CUDA / TR_ERR_NOMEM.
+ *   (malformed tree, n_nodes > TR_MAX_NODES), TR_ERR_UNSUPPORTED (batch * n_nodes > 65535), TR_ERR_CUDA / TR_ERR_NOMEM.
  */
 tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32_t* parent, const int32_t* rank,
                   int32_t n_nodes, int32_t batch, int32_t device);
@@ -76,6 +76,18 @@ tr_status tr_destroy(tr_ctx* ctx); /* frees everything tr_init allocated; synchr
 
 /* Matrix state (Sec. 3.1: zero initialisation, or "hot start" = keep / restore an earlier matrix). */
 tr_status tr_matrix_zero(tr_ctx* ctx, void* stream);                                /* all sequences */
+/*
+ * Fill all sequences' matrices on the device (Sec. 5.2, study of initialisations: zeros, or random token ids).
+ *   TR_FILL_ZERO   : every entry 0 (= tr_matrix_zero)
+ *   TR_FILL_SEEDED : entry number i of the context's [batch, V, k] array (i = (b * V + token) * k + column) is
+ *                    (hi32(mix(seed + 0x9E3779B97F4A7C15 * (i + 1))) * V) >> 32, where mix is the splitmix64 finaliser
+ *                    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9; z ^= z >> 27; z *= 0x94D049BB133111EB; z ^= z >> 31
+ *                    (64-bit wrap-around arithmetic) - uniform token ids in [0, V), reproducible on any host.
+ * Errors: TR_ERR_INVALID_ARG (NULL, unknown mode).  Does not synchronise.
+ */
+#define TR_FILL_ZERO 0
+#define TR_FILL_SEEDED 1
+tr_status tr_matrix_fill(tr_ctx* ctx, int32_t mode, uint64_t seed, void* stream);
 tr_status tr_matrix_import(tr_ctx* ctx, int32_t seq, const int32_t* host_M);        /* HOST [V*k]; synchronises */
 tr_status tr_matrix_export(tr_ctx* ctx, int32_t seq, int32_t* host_M);              /* HOST [V*k]; synchronises */
 int32_t* tr_matrix_device_ptr(tr_ctx* ctx, int32_t seq);                            /* DEVICE, borrowed; NULL on error */
@@ -150,7 +162,9 @@ int32_t tr_max_new_tokens(const tr_ctx* ctx); /* depth of the template + 1 (Appe
 /*
  * The same step from a top-k that is already on the device (for example from tr_lm_head_topk): everything
  * tr_verify_update does after its argtopk.  out->d_topk_idx [batch, N, k] is an INPUT here (indices in [0, V),
- * column 0 the argmax); the other members of `out` are written as by tr_verify_update.
+ * column 0 the argmax); the other members of `out` are written as by tr_verify_update.  An index outside [0, V)
+ * sets TR_FLAG_BAD_TOKEN and is treated as token 0 (the matrix never holds an id outside the vocabulary).
+ * d_tree and d_topk_idx may have been written by the kernel directly in front on the same stream.
  */
 tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream);
 
@@ -198,18 +212,23 @@ tr_status tr_lm_head_topk(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stri
  * "Explanation of Three Update Strategies").  Takes effect for the following tr_verify_update calls.
  *   rule : TR_UPDATE_LAST  (default) - a repeated token keeps the row of its last occurrence
  *          TR_UPDATE_FIRST           - ... of its first occurrence
+ *          TR_UPDATE_CUR             - the paper's own uncontrolled update: every occurrence stores its row, one 32-bit
+ *                                      element at a time, with nothing ordering the occurrences - each element of a
+ *                                      repeated token's row ends up as that element of ONE of its occurrences, and
+ *                                      different elements may come from different occurrences; not reproducible
+ *                                      from run to run (rows of tokens that occur once are as under the other rules)
  *   scope: TR_UPDATE_ALL_DRAFT (default) - every node of the tree updates its token's row
  *          TR_UPDATE_ONLY_ACCEPTED       - only the nodes of the accepted path do
- * The paper's own uncontrolled update ("Cur") is a data race by design and is not offered.
  */
 #define TR_UPDATE_LAST 0
 #define TR_UPDATE_FIRST 1
+#define TR_UPDATE_CUR 2
 #define TR_UPDATE_ALL_DRAFT 0
 #define TR_UPDATE_ONLY_ACCEPTED 1
 tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope);
 
 /*
- * Commit the accepted path (Sec. 5.4: a step ends by "updating the matrix, input tokens, and key-value cache").
+ * Commit the accepted path (Sec. 5.4: besides the matrix, a step also advances the token list and the KV cache).
  * Call after tr_verify_update with its outputs.  For every sequence b with n = n_new[b] and accepted nodes
  * a_0 = 0 (root), a_1, ..., a_{n-1} (acc_nodes[b]):
  *   K/V : for every layer and KV head, cache row C_b + a_i moves to row C_b + i (i = 1..n-1; the root's row is in
@@ -247,7 +266,8 @@ tr_status tr_device_flags(tr_ctx* ctx, uint32_t* host_flags);
  * runs tr_tree_attention over n_layers layers, then tr_verify_update, copies the results back and waits.
  * The prefix K/V (rows [0, C_b)) and the current tree stay resident in device buffers the caller owns.
  * HOST in : h_q [batch, L, N, Hq, D] bf16; h_tree_k / h_tree_v [batch, L, Hkv, N, D] bf16 (this step's tree
- *           rows, written to cache rows C_b..C_b+N-1; h_ctx_len[batch] gives C_b); h_logits [batch, N, V] fp32.
+ *           rows, written to cache rows C_b..C_b+N-1; h_ctx_len[batch] gives C_b and is copied to a->d_ctx_len, the
+ *           device array the attention kernel reads, at the start of the call); h_logits [batch, N, V] fp32.
  * DEVICE  : a->q / a->out must be buffers of that shape (used as staging), a->k_cache / a->v_cache the caches
  *           with kv_stride/layer_stride_kv as described above; d_logits_staging [batch,N,V]; d_tree [batch,N]
  *           current tree (updated in place to the next tree); d_out as in tr_verify_update.
@@ -282,9 +302,10 @@ tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_step_out* d_
  * callers cannot hold a context; this function needs none.
  *
  * What it computes: exactly the top-k part of tr_verify_update - for each of `rows` logits rows the indices of the
- * k largest values, largest first, equal values by lower index (Sec. 2.1) - with the same kernel.  Its scratch
- * (per-segment candidate lists and per-row tickets) lives in a fixed 528 KB device array inside the library,
- * held by every GPU that loads the library until the process exits.
+ * k largest values, largest first, equal values by lower index - with a kernel that cuts every row into segments of
+ * 4096 values, keeps per-segment candidate lists in scratch memory and lets the last CTA of a row (a per-row ticket)
+ * merge them.  That scratch lives in a fixed 528 KB device array inside the library, held by every GPU that loads the
+ * library until the process exits.
  * DEVICE in : d_logits [rows, vocab] fp32 row-major.   DEVICE out: d_topk_idx [rows, k] int32.
  * Limits    : rows <= 4096 and rows * ceil(vocab / 4096) * k <= 65536 (tr_topk_noalloc_limits reports both);
  *             anything larger returns TR_ERR_UNSUPPORTED and launches nothing.  1 <= k <= TR_MAX_K <= vocab.

@@ -337,7 +337,7 @@ def verify_update_sampled(M, S, logits, gumbel, inv_temperature, parent, rank, r
 
 
 # --------------------------------------------------------------------------
-# Commit of the accepted path (Sec. 5.4: "updating the matrix, input tokens, and key-value cache")
+# Commit of the accepted path (Sec. 5.4: besides the matrix, a step advances the token list and the KV cache)
 # --------------------------------------------------------------------------
 def commit(k, v, ctx_len, tokens, acc_nodes, out_tokens):
     """After verification the accepted nodes (root first) are the tokens whose keys and values now belong to the

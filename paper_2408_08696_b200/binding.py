@@ -13,7 +13,7 @@ import numpy as np
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_TR_PATH = os.environ.get("TR_LIB_PATH") or os.path.join(_PKG, "libtr.so")  # override: debugging aid
+LIB_TR_PATH = os.path.join(_PKG, "libtr.so")
 LIB_SYNTH_PATH = os.path.join(_PKG, "libtr_synth.so")
 
 if not os.path.exists(LIB_TR_PATH) or not os.path.exists(LIB_SYNTH_PATH):
@@ -28,7 +28,8 @@ TR_OK = 0
 TR_ERR_INVALID_ARG, TR_ERR_TEMPLATE, TR_ERR_UNSUPPORTED, TR_ERR_CUDA, TR_ERR_NOMEM, TR_ERR_DEVICE_FLAG = -1, -2, -3, -4, -5, -6
 TR_FLAG_BAD_TOKEN, TR_FLAG_WAIT_TIMEOUT, TR_FLAG_CACHE_FULL = 1, 2, 4
 TR_MAX_NODES, TR_MAX_K = 128, 16
-TR_UPDATE_LAST, TR_UPDATE_FIRST, TR_UPDATE_ALL_DRAFT, TR_UPDATE_ONLY_ACCEPTED = 0, 1, 0, 1
+TR_UPDATE_LAST, TR_UPDATE_FIRST, TR_UPDATE_CUR, TR_UPDATE_ALL_DRAFT, TR_UPDATE_ONLY_ACCEPTED = 0, 1, 2, 0, 1
+TR_FILL_ZERO, TR_FILL_SEEDED = 0, 1
 
 
 class TrError(RuntimeError):
@@ -76,6 +77,7 @@ lib.tr_template_from_branching.argtypes = [_P32, C.c_int32, C.c_int32, _P32, _P3
 lib.tr_init.argtypes = [C.POINTER(C.c_void_p), C.c_int32, C.c_int32, _P32, _P32, C.c_int32, C.c_int32, C.c_int32]
 lib.tr_destroy.argtypes = [C.c_void_p]
 lib.tr_matrix_zero.argtypes = [C.c_void_p, C.c_void_p]
+lib.tr_matrix_fill.argtypes = [C.c_void_p, C.c_int32, C.c_uint64, C.c_void_p]
 lib.tr_matrix_import.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
 lib.tr_matrix_export.argtypes = [C.c_void_p, C.c_int32, C.c_void_p]
 lib.tr_matrix_device_ptr.restype = C.c_void_p
@@ -170,6 +172,11 @@ def tr_destroy(ctx):
 
 def tr_matrix_zero(ctx, stream=None):
     _check(lib.tr_matrix_zero(ctx.handle, _stream(stream)), "tr_matrix_zero")
+
+
+def tr_matrix_fill(ctx, mode, seed=0, stream=None):
+    _check(lib.tr_matrix_fill(ctx.handle, int(mode), C.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _stream(stream)),
+           "tr_matrix_fill")
 
 
 def tr_matrix_import(ctx, seq, host_M):

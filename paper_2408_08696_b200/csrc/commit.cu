@@ -1,4 +1,4 @@
-// Commit of the accepted path (paper Sec. 5.4: "updating the matrix, input tokens, and key-value cache"): the
+// Commit of the accepted path (paper Sec. 5.4: besides the matrix, a step advances the token list and the KV cache): the
 // accepted nodes' K/V rows are compacted to the end of the prefix, the confirmed tokens are appended, the prefix
 // length grows - all on the device, so the step graph replays without the host.
 //

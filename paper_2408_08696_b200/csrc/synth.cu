@@ -22,8 +22,9 @@ extern "C" int32_t trs_patch_logits(float* d_logits, const float* d_noise, const
                                     int32_t* d_prev_col, const int32_t* d_succ, float boost, int32_t rows,
                                     int32_t V, void* stream) {
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3((rows + 127) / 128);
-  cfg.blockDim = dim3(128);
+  // one warp per CTA: small enough to slip onto an SM beside a resident CTA of a large kernel running concurrently
+  cfg.gridDim = dim3((rows + 31) / 32);
+  cfg.blockDim = dim3(32);
   cfg.stream = static_cast<cudaStream_t>(stream);
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

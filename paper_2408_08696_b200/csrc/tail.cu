@@ -6,7 +6,8 @@
 //            walks its own path (<= depth_max steps); the deepest correct node, lowest index among equals, is
 //            found with one packed-key maximum (warp reduce + shared memory).
 //   update : M[S[i]] <- topk[i] for all i; when a token repeats, only the highest i writes, which is what the
-//            sequential loop "for i: M[S[i]] = O[i]" leaves behind - deterministic, no write races.
+//            sequential loop "for i: M[S[i]] = O[i]" leaves behind - deterministic, no write races.  (TR_UPDATE_CUR,
+//            the paper's uncontrolled update, lets every occurrence store its row element by element instead.)
 //   BFS    : S'[0] = argmax[last accepted]; level by level S'[i] = M[S'[parent i]][rank i], reading the rows
 //            written a moment ago by this same CTA (ordered by __syncthreads()).
 #include "tr_internal.cuh"
@@ -74,7 +75,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
                const int32_t* __restrict__ topk_idx, int32_t* __restrict__ n_new, int32_t* __restrict__ acc_nodes,
                int32_t* __restrict__ out_tokens, int32_t* __restrict__ next_root, int32_t* tree_out,
                uint32_t* __restrict__ flags, const uint32_t* __restrict__ anc, int update_rule, int update_scope,
-               const int32_t* __restrict__ target) {
+               const int32_t* __restrict__ target, int tree_early) {
   __shared__ int32_t s_S[TR_MAX_NODES];
   __shared__ int32_t s_argmax[TR_MAX_NODES];  // the token each node's children must match: argmax, or the given draw
   __shared__ int32_t s_tree[TR_MAX_NODES];
@@ -86,20 +87,36 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   const int32_t* topk = topk_idx + static_cast<size_t>(b) * n * k;
   const int W = depth_max + 1;
 
+  // the kernel behind this one may be scheduled now; it must wait for this grid before it reads anything written here
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   int32_t tok = 0;
   int32_t row[TR_MAX_K];
   bool tok_ok = false;
-  if (tid < n) tok = tree_in[static_cast<size_t>(b) * n + tid];  // written by an earlier step, not by the top-k kernel
-  // Everything above was fetched while the top-k kernel may still have been running (programmatic dependent
+  // tree_early: the tree was written at least two kernels back on this stream (tr_verify_update: the top-k kernel sits
+  // in between and has itself waited for its predecessor), so it may be fetched while the top-k kernel is still running
+  if (tree_early && tid < n) tok = tree_in[static_cast<size_t>(b) * n + tid];
+  // Everything above was fetched while the kernel in front may still have been running (programmatic dependent
   // launch); its output is read only from here on.
   tr_grid_dependency_wait();
   if (tid < n) {
+    if (!tree_early) tok = tree_in[static_cast<size_t>(b) * n + tid];
     tok_ok = (tok >= 0 && tok < V);
-    if (!tok_ok) atomicOr(flags, TR_FLAG_BAD_TOKEN);
+    bool ids_ok = tok_ok;
     s_S[tid] = tok;
+    // the candidates are stored into M and later used as row indices: anything outside [0, V) is replaced by token 0
 #pragma unroll
-    for (int c = 0; c < TR_MAX_K; ++c) row[c] = c < k ? topk[tid * k + c] : 0;  // fetched once, with the tokens
-    s_argmax[tid] = target ? target[static_cast<size_t>(b) * n + tid] : row[0];
+    for (int c = 0; c < TR_MAX_K; ++c) {
+      int32_t x = c < k ? topk[tid * k + c] : 0;  // fetched once, with the tokens
+      if (x < 0 || x >= V) { x = 0; ids_ok = false; }
+      row[c] = x;
+    }
+    int32_t want = row[0];
+    if (target) {
+      want = target[static_cast<size_t>(b) * n + tid];
+      if (want < 0 || want >= V) { want = 0; ids_ok = false; }
+    }
+    s_argmax[tid] = want;
+    if (!ids_ok) atomicOr(flags, TR_FLAG_BAD_TOKEN);
   }
   __syncthreads();
 
@@ -156,9 +173,9 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
     bool last = true;
     if (update_rule == TR_UPDATE_FIRST) {
       for (int j = 0; j < tid; ++j) last = last && (s_S[j] != tok);
-    } else {
+    } else if (update_rule == TR_UPDATE_LAST) {
       for (int j = tid + 1; j < n; ++j) last = last && (s_S[j] != tok);
-    }
+    }  // TR_UPDATE_CUR: every occurrence stores; the 32-bit stores of different occurrences land in any order
     if (last) {
       int32_t* dst = M + static_cast<size_t>(tok) * k;
 #pragma unroll
@@ -180,11 +197,11 @@ tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tr
 }
 
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s,
-                         const int32_t* d_target) {
+                         const int32_t* d_target, bool tree_early) {
   TR_CUDA_TRY(tr_launch_pdl(tr_tail_kernel, dim3(ctx->batch), dim3(TAIL_THREADS), 0, s, ctx->d_M, ctx->vocab, ctx->k,
                             ctx->n_nodes, ctx->d_parent, ctx->d_rank, ctx->d_depth, ctx->d_level_off, ctx->depth_max,
                             d_tree, out->d_topk_idx, out->d_n_new, out->d_acc_nodes, out->d_out_tokens,
                             out->d_next_root, out->d_next_tree, ctx->d_flags, ctx->d_anc, ctx->update_rule,
-                            ctx->update_scope, d_target));
+                            ctx->update_scope, d_target, tree_early ? 1 : 0));
   return TR_OK;
 }

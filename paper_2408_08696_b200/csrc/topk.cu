@@ -1,315 +1,273 @@
 // Fused per-node argmax + top-k over fp32 vocabulary logits (paper Sec. 2.1: argtopk, x^0 = argmax).
 //
-// Order: value descending, equal values by lower index.  Every (value, index) pair is packed into one
-// 64-bit key whose unsigned order IS that order, so all keys are distinct and "top-k" means "the k largest
-// keys" - any split / merge order gives the same answer, bit for bit.
+// Order: value descending, equal values by lower index.  Every (value, index) pair is packed into one 64-bit key
+// whose unsigned order IS that order, so all keys are distinct and "top-k" means "the k largest keys" - any split /
+// merge order gives the same answer, bit for bit.
 //
-// A logits row is cut into segments of TOPK_SEG_ELEMS; one CTA per (segment, row) keeps its 16 values per
-// thread in registers (128-bit loads), finds a threshold that cannot exceed the segment's k-th largest key
-// (the k-th largest of the 16 half-warp maxima), collects the few keys at or above it - only threads whose own
-// maximum reaches the threshold look at all - and selects the segment's top-k exactly.  The last CTA of a row
-// to finish (atomic ticket, no waiting) merges the per-segment lists into the row's final top-k.
+// One thread-block cluster per logits row, P = 1, 2, 4 or 8 CTAs; CTA p scans a contiguous part of the row in chunks
+// of 4096 values (16 per thread in registers, 128-bit streaming loads).  The hot loop works on the float values only:
+//   threshold : tau = k-th largest of the chunk's 16 half-warp maxima (at least k values of the part are >= tau, so
+//               the part's k best keys are among the values >= tau); tau only grows from chunk to chunk
+//   candidates: the few values >= tau are turned into keys and pushed to shared memory (threads whose own maximum is
+//               below tau skip the scan)
+//   part list : candidates ranked by counting -> the part's k best keys, stored straight into the shared memory of
+//               the cluster's first CTA (distributed shared memory)
+//   merge     : after one cluster barrier the first CTA ranks the P * k keys by counting and writes the row's top-k.
+// No global scratch, no atomics on global memory, no second kernel.  Massive ties (more candidates than the buffer
+// holds) take an exact, slower path that selects round by round from global memory.
 #include "tr_internal.cuh"
 
+namespace {
+
 typedef unsigned long long u64;
-constexpr int TOPK_MERGE_CAP = 1024;
-constexpr int TOPK_CAND_CAP = 512;
+constexpr int CHUNK = TOPK_SEG_ELEMS;        // values per CTA and iteration
+constexpr int E = TOPK_ELEMS_PER_THREAD;     // values per thread and iteration
+constexpr int CAND_CAP = 512;
+constexpr int MAX_PARTS = 8;
 
-__device__ __forceinline__ u64 topk_key(float v, uint32_t idx) {
+// float -> uint32 whose unsigned order is the float order (-0 and +0 coincide), and back
+__device__ __forceinline__ uint32_t ord_u32(float v) {
   uint32_t b = __float_as_uint(v);
-  if (b == 0x80000000u) b = 0u;  // -0 and +0 compare equal: the index decides
-  const uint32_t s = (b & 0x80000000u) ? ~b : (b | 0x80000000u);
-  return (static_cast<u64>(s) << 32) | static_cast<u64>(0xFFFFFFFFu - idx);
+  if (b == 0x80000000u) b = 0u;
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
-
+__device__ __forceinline__ float ord_to_float(uint32_t s) {
+  return __uint_as_float((s & 0x80000000u) ? (s ^ 0x80000000u) : ~s);
+}
+__device__ __forceinline__ u64 topk_key(float v, uint32_t idx) {
+  return (static_cast<u64>(ord_u32(v)) << 32) | static_cast<u64>(0xFFFFFFFFu - idx);
+}
 __device__ __forceinline__ u64 warp_max_u64(u64 x) {
   const uint32_t hi = static_cast<uint32_t>(x >> 32), lo = static_cast<uint32_t>(x);
   const uint32_t mh = __reduce_max_sync(0xFFFFFFFFu, hi);
   const uint32_t ml = __reduce_max_sync(0xFFFFFFFFu, hi == mh ? lo : 0u);
   return (static_cast<u64>(mh) << 32) | ml;
 }
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+// store into the shared memory of the cluster's CTA 0 (same offset as the local address `p`)
+__device__ __forceinline__ void st_leader_u64(const void* p, u64 v) {
+  const uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(p));
+  uint32_t remote;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0u));
+  asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+}
 
 // kSample: rank z = fl32(fl32(logit * inv_t) + gumbel) instead of the logits (Sec. 5.3 temperature sampling: with k = 1
 // the result is the token drawn at temperature 1 / inv_t by the Gumbel-max rule).  Two roundings, no fused multiply-add:
 // the decision is reproducible with plain float32 arithmetic.
-template <bool kVec, bool kSample = false>
-__global__ void __launch_bounds__(TOPK_THREADS, 5)
-tr_topk_kernel(const float* __restrict__ logits, int V, int k, int segs, u64* __restrict__ part,
-               unsigned int* __restrict__ ticket, int32_t* __restrict__ topk_idx,
-               const float* __restrict__ gumbel = nullptr, float inv_t = 1.f) {
-  constexpr int E = TOPK_ELEMS_PER_THREAD;
-  constexpr int G = TOPK_THREADS / 16;  // half-warp groups: 16 >= TR_MAX_K
-  __shared__ u64 s_gmax[G];
-  __shared__ u64 s_cand[TOPK_CAND_CAP];
-  __shared__ u64 s_out[TR_MAX_K];
-  __shared__ u64 s_merge[TOPK_MERGE_CAP];
-  __shared__ u64 s_tau;
+template <bool kVec, bool kSample>
+__global__ void __launch_bounds__(TOPK_THREADS)
+tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_part, int32_t* __restrict__ topk_idx,
+               const float* __restrict__ gumbel, float inv_t) {
+  __shared__ u64 s_cand[CAND_CAP];
+  __shared__ u64 s_all[MAX_PARTS * TR_MAX_K];  // CTA 0 of the cluster: every part's list
+  __shared__ u64 s_red[TOPK_THREADS / 32];
+  __shared__ uint32_t s_gmax[2][16];
   __shared__ int s_cnt;
-  __shared__ int s_last;
 
-  const int seg = blockIdx.x;
-  const int row = blockIdx.y;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int part = blockIdx.x, P = gridDim.x, row = blockIdx.y;
+  const int tid = threadIdx.x, lane = tid & 31;
   const float* rowp = logits + static_cast<size_t>(row) * V;
-  const int seg_base = seg * TOPK_SEG_ELEMS;
+  const float* rowg = kSample ? gumbel + static_cast<size_t>(row) * V : nullptr;
+  const int part_base = part * chunks_per_part * CHUNK;
+  const int part_end = min(V, part_base + chunks_per_part * CHUNK);
+
+  if (tid == 0) s_cnt = 0;
+  // first half of a cluster barrier: before a CTA stores into the first CTA's shared memory (below), every CTA of the
+  // cluster must have started
+  if (P > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
   // (programmatic dependent launch) the logits belong to whatever ran before on this stream
   tr_grid_dependency_wait();
+  // The kernel behind this one (accept / update / retrieve) may be scheduled from here on and run its preamble; it
+  // waits for this grid to finish before it reads the result.  (Only after the wait above: whatever that kernel
+  // fetches early must come from kernels that are complete by now.)
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
-  // ---- (1) 16 values per thread in registers; running maximum with its index (first = lowest index wins ties)
-  float v[E];
-  int idx0[E / 4];  // index of each 4-group's first element (vector path) -- scalar path uses j * THREADS + tid
-  if (kVec) {
-#pragma unroll
-    for (int j = 0; j < E / 4; ++j) {
-      const int i0 = seg_base + j * (TOPK_THREADS * 4) + tid * 4;
-      idx0[j] = i0;
-      float4 t = (i0 < V) ? __ldcs(reinterpret_cast<const float4*>(rowp + i0))
-                          : make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
-      if (kSample && i0 < V) {
-        const float4 g = __ldcs(reinterpret_cast<const float4*>(gumbel + static_cast<size_t>(row) * V + i0));
-        t.x = __fadd_rn(__fmul_rn(t.x, inv_t), g.x); t.y = __fadd_rn(__fmul_rn(t.y, inv_t), g.y);
-        t.z = __fadd_rn(__fmul_rn(t.z, inv_t), g.z); t.w = __fadd_rn(__fmul_rn(t.w, inv_t), g.w);
-      }
-      v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
-    }
-  } else {
-#pragma unroll
-    for (int j = 0; j < E; ++j) {
-      const int i = seg_base + j * TOPK_THREADS + tid;
-      v[j] = (i < V) ? __ldcs(rowp + i) : -INFINITY;
-      if (kSample && i < V) v[j] = __fadd_rn(__fmul_rn(v[j], inv_t), __ldcs(gumbel + static_cast<size_t>(row) * V + i));
-    }
-  }
-  auto index_of = [&](int j) -> int {
-    return kVec ? idx0[j >> 2] + (j & 3) : seg_base + j * TOPK_THREADS + tid;
+  auto index_of = [&](int base, int j) -> int {
+    return kVec ? base + (j >> 2) * (TOPK_THREADS * 4) + tid * 4 + (j & 3) : base + j * TOPK_THREADS + tid;
   };
-  if (tid == 0) s_cnt = 0;
-  float bv = v[0];
-  int bj = 0;
+  auto load_chunk = [&](int base, float (&v)[E]) {
+    if (kVec) {
 #pragma unroll
-  for (int j = 1; j < E; ++j)
-    if (v[j] > bv) { bv = v[j]; bj = j; }  // -0 == +0 here as well; indices ascend with j
-  int bi = 0;
+      for (int j = 0; j < E / 4; ++j) {
+        const int i0 = base + j * (TOPK_THREADS * 4) + tid * 4;
+        float4 t = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        if (i0 < part_end) {
+          t = __ldcs(reinterpret_cast<const float4*>(rowp + i0));
+          if (kSample) {
+            const float4 g = __ldcs(reinterpret_cast<const float4*>(rowg + i0));
+            t.x = __fadd_rn(__fmul_rn(t.x, inv_t), g.x); t.y = __fadd_rn(__fmul_rn(t.y, inv_t), g.y);
+            t.z = __fadd_rn(__fmul_rn(t.z, inv_t), g.z); t.w = __fadd_rn(__fmul_rn(t.w, inv_t), g.w);
+          }
+        }
+        v[4 * j] = t.x; v[4 * j + 1] = t.y; v[4 * j + 2] = t.z; v[4 * j + 3] = t.w;
+      }
+    } else {
 #pragma unroll
-  for (int j = 0; j < E; ++j) bi = (bj == j) ? index_of(j) : bi;
-  const u64 tmax = (bi < V) ? topk_key(bv, bi) : 0ull;  // padding threads past the row's end hold no key
-
-  // ---- (2) maxima of the 16 half-warp groups; threshold = k-th largest of them.  At least k keys of the segment
-  //          are >= it, so the segment's top-k lies among the keys >= it.
-  {
-    const unsigned mask = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
-    const uint32_t hi = static_cast<uint32_t>(tmax >> 32), lo = static_cast<uint32_t>(tmax);
-    const uint32_t mh = __reduce_max_sync(mask, hi);
-    const uint32_t ml = __reduce_max_sync(mask, hi == mh ? lo : 0u);
-    if ((lane & 15) == 0) s_gmax[tid >> 4] = (static_cast<u64>(mh) << 32) | ml;
-  }
-  __syncthreads();
-  // rank by counting, by half a warp for the whole CTA: the group maximum that has exactly k-1 larger ones is the
-  // threshold; with fewer than k non-empty groups the threshold is 0 and every key is a candidate
-  if (warp == 0) {
-    const u64 mine = lane < G ? s_gmax[lane] : 0ull;
-    int larger = 0;
-#pragma unroll
-    for (int i = 0; i < G; ++i) larger += (s_gmax[i] > mine) ? 1 : 0;
-    const unsigned hit = __ballot_sync(0xFFFFFFFFu, lane < G && mine != 0ull && larger == k - 1);
-    if (hit == 0u) {
-      if (lane == 0) s_tau = 0ull;
-    } else if (lane == __ffs(hit) - 1) {
-      s_tau = mine;
+      for (int j = 0; j < E; ++j) {
+        const int i = base + j * TOPK_THREADS + tid;
+        float x = -INFINITY;
+        if (i < part_end) {
+          x = __ldcs(rowp + i);
+          if (kSample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcs(rowg + i));
+        }
+        v[j] = x;
+      }
     }
-  }
-  __syncthreads();
-  const u64 tau = s_tau;
-  // ---- (3) candidates: only threads whose own maximum reaches the threshold look at their values
-  if (tmax != 0 && tmax >= tau) {
-    const uint32_t tau_hi = static_cast<uint32_t>(tau >> 32);
+  };
+
+  // ---- scan the part chunk by chunk; the next chunk's loads are in flight while the current one is examined
+  uint32_t tau_ord = 0u;  // below every value, -inf included
+  float v[E], vn[E];
+  if (part_base < part_end) load_chunk(part_base, v);
+  for (int c = 0; c < chunks_per_part; ++c) {
+    const int base = part_base + c * CHUNK;
+    if (base >= part_end) break;  // uniform over the CTA
+    const bool more = (c + 1 < chunks_per_part) && (base + CHUNK < part_end);
+    if (more) load_chunk(base + CHUNK, vn);
+    // thread maximum (values only: -0 == +0, no NaN by precondition), then the maxima of the 16 half-warp groups
+    float m = max3f(v[0], v[1], v[2]);
 #pragma unroll
-    for (int j = 0; j < E; ++j) {
-      const int i = index_of(j);
-      // cheap filter on the value alone, then the exact (value, index) comparison
-      if (i < V && static_cast<uint32_t>(topk_key(v[j], 0u) >> 32) >= tau_hi) {
-        const u64 key = topk_key(v[j], i);
-        if (key >= tau) {
-          const int p = atomicAdd(&s_cnt, 1);
-          if (p < TOPK_CAND_CAP) s_cand[p] = key;
+    for (int j = 3; j + 1 < E; j += 2) m = max3f(m, v[j], v[j + 1]);
+    m = fmaxf(m, v[E - 1]);
+    {
+      const unsigned mask = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
+      const uint32_t gm = __reduce_max_sync(mask, ord_u32(m));
+      if ((lane & 15) == 0) s_gmax[c & 1][tid >> 4] = gm;
+    }
+    __syncthreads();
+    // every warp works the threshold out for itself: the group maximum with fewer than k larger and at least k
+    // larger-or-equal ones is the k-th largest.  Groups past the row's end hold -inf; with fewer than k real groups
+    // the threshold is -inf and every value of the chunk is a candidate.
+    {
+      const uint32_t mine = s_gmax[c & 1][lane & 15];
+      int larger = 0, ge = 0;
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const uint32_t g = s_gmax[c & 1][i];
+        larger += (g > mine) ? 1 : 0;
+        ge += (g >= mine) ? 1 : 0;
+      }
+      const unsigned hit = __ballot_sync(0xFFFFFFFFu, larger < k && ge >= k);
+      const uint32_t tau_c = hit ? __shfl_sync(0xFFFFFFFFu, mine, __ffs(hit) - 1) : 0u;  // k <= 16 groups: always a hit
+      tau_ord = max(tau_ord, tau_c);
+    }
+    const float tau = ord_to_float(tau_ord);
+    if (m >= tau) {
+#pragma unroll
+      for (int j = 0; j < E; ++j) {
+        if (v[j] >= tau) {
+          const int i = index_of(base, j);
+          if (i < part_end) {
+            const int p = atomicAdd(&s_cnt, 1);
+            if (p < CAND_CAP) s_cand[p] = topk_key(v[j], i);
+          }
         }
       }
     }
+    if (more) {
+#pragma unroll
+      for (int j = 0; j < E; ++j) v[j] = vn[j];
+    }
   }
   __syncthreads();
-  // ---- (4) exact top-k of the candidates -> this segment's partial list
-  u64* my_part = part + (static_cast<size_t>(row) * segs + seg) * k;
+
+  // ---- the part's k best keys -> list `part` in the first CTA's shared memory (unused entries are 0)
+  u64* my_list = s_all + part * TR_MAX_K;
   const int cnt = s_cnt;
-  if (cnt <= TOPK_CAND_CAP) {
-    // rank by counting: candidate with r larger ones is the segment's r-th entry; unused entries are 0
+  if (P > 1) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
+  if (cnt <= CAND_CAP) {
     for (int t = tid; t < cnt; t += TOPK_THREADS) {
       const u64 mine = s_cand[t];
       int larger = 0;
       for (int i = 0; i < cnt; ++i) larger += (s_cand[i] > mine) ? 1 : 0;
-      if (larger < k) my_part[larger] = mine;
+      if (larger < k) st_leader_u64(my_list + larger, mine);
     }
-    if (tid >= cnt && tid < k) my_part[tid] = 0ull;
-    // (these writes are published by the barrier below together with thread 0's fence, which is cumulative)
+    if (tid >= cnt && tid < k) st_leader_u64(my_list + tid, 0ull);
   } else {
-    // More candidates than the buffer holds (only with massive ties or adversarial layouts): select straight
-    // from the registers, round by round, the whole CTA taking part.
+    // More candidates than the buffer holds (massive ties or adversarial layouts): select straight from global
+    // memory, round by round, the whole CTA taking part.
     u64 last = ~0ull;
     for (int r = 0; r < k; ++r) {
       u64 best = 0;
-#pragma unroll
-      for (int j = 0; j < E; ++j) {
-        const int i = index_of(j);
-        const u64 key = (i < V) ? topk_key(v[j], i) : 0ull;
+      for (int i = part_base + tid; i < part_end; i += TOPK_THREADS) {
+        float x = __ldcg(rowp + i);
+        if (kSample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcg(rowg + i));
+        const u64 key = topk_key(x, i);
         if (key < last && key > best) best = key;
       }
       best = warp_max_u64(best);
-      __syncthreads();  // previous round's readers are done with s_gmax
-      if (lane == 0) s_gmax[warp] = best;
+      __syncthreads();  // the previous round's readers are done with s_red
+      if (lane == 0) s_red[tid >> 5] = best;
       __syncthreads();
-      u64 m = 0;
+      u64 mx = 0;
 #pragma unroll
-      for (int w = 0; w < TOPK_THREADS / 32; ++w) m = s_gmax[w] > m ? s_gmax[w] : m;
-      last = m;
-      if (tid == 0) my_part[r] = m;
+      for (int w = 0; w < TOPK_THREADS / 32; ++w) mx = s_red[w] > mx ? s_red[w] : mx;
+      last = mx;
+      if (tid == 0) st_leader_u64(my_list + r, mx);
     }
   }
-  // ---- (5) ticket: the last CTA of the row merges all partial lists
-  __syncthreads();
-  if (tid == 0) {
-    __threadfence();
-    const unsigned int t = atomicAdd(&ticket[row], 1u);
-    s_last = (t == static_cast<unsigned int>(segs - 1));
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  const u64* row_part = part + static_cast<size_t>(row) * segs * k;
-  const int n = segs * k;
-  const bool staged = n <= TOPK_MERGE_CAP;  // one parallel fetch of every partial list, then rounds in shared memory
-  if (staged) {
-    for (int i = tid; i < n; i += TOPK_THREADS) s_merge[i] = __ldcg(row_part + i);
+
+  // ---- merge in the cluster's first CTA
+  if (P > 1) {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    if (part != 0) return;  // the lists are delivered; only the first CTA goes on
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  } else {
     __syncthreads();
   }
-  if (staged) {
-    // every partial key counts the keys above it; the k keys with fewer than k above them are the answer
-    for (int t = tid; t < n; t += TOPK_THREADS) {
-      const u64 mine = s_merge[t];
-      if (mine == 0ull) continue;
+  const int n = P * TR_MAX_K;
+  if (tid < n && (tid & (TR_MAX_K - 1)) < k) {
+    const u64 mine = s_all[tid];
+    if (mine != 0ull) {
       int larger = 0;
-      for (int i = 0; i < n; ++i) larger += (s_merge[i] > mine) ? 1 : 0;
+      for (int q = 0; q < P; ++q)
+        for (int i = 0; i < k; ++i) larger += (s_all[q * TR_MAX_K + i] > mine) ? 1 : 0;
       if (larger < k)
         topk_idx[static_cast<size_t>(row) * k + larger] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(mine));
     }
-    if (tid == 0) ticket[row] = 0u;  // ready for the next launch
-  } else if (warp == 0) {
-    u64 last = ~0ull;
-    for (int r = 0; r < k; ++r) {
-      u64 best = 0;
-      for (int i = lane; i < n; i += 32) {
-        const u64 x = __ldcg(row_part + i);
-        if (x < last && x > best) best = x;
-      }
-      last = warp_max_u64(best);
-      if (lane == 0) s_out[r] = last;
-    }
-    __syncwarp();
-    if (lane < k) topk_idx[static_cast<size_t>(row) * k + lane] =
-        static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(s_out[lane]));
-    if (lane == 0) ticket[row] = 0u;
   }
 }
+
+}  // namespace
 
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
                          const float* d_gumbel, float inv_temperature, int k_override) {
   const int rows = ctx->batch * ctx->n_nodes;
   const int k = k_override > 0 ? k_override : ctx->k;
-  dim3 grid(ctx->topk_segs, rows);
+  const int chunks = (ctx->vocab + CHUNK - 1) / CHUNK;
+  int P = 1;
+  while (P < MAX_PARTS && P < chunks) P *= 2;
+  const int cpp = (chunks + P - 1) / P;
   bool vec = (ctx->vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
-  if (d_gumbel) {
-    vec = vec && ((reinterpret_cast<uintptr_t>(d_gumbel) & 15) == 0);
-    if (vec)
-      TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true, true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
-                                ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, d_gumbel,
-                                inv_temperature));
-    else
-      TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false, true>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
-                                ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, d_gumbel,
-                                inv_temperature));
-    return TR_OK;
-  }
-  const float* no_noise = nullptr;
-  if (vec)
-    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<true, false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
-                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, no_noise, 1.f));
+  if (d_gumbel) vec = vec && ((reinterpret_cast<uintptr_t>(d_gumbel) & 15) == 0);
+
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(P, rows);
+  cfg.blockDim = dim3(TOPK_THREADS);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = P;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  const int V = ctx->vocab;
+  cudaError_t e;
+  if (d_gumbel)
+    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, inv_temperature)
+            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, inv_temperature);
   else
-    TR_CUDA_TRY(tr_launch_pdl(tr_topk_kernel<false, false>, grid, dim3(TOPK_THREADS), 0, s, d_logits, ctx->vocab, k,
-                              ctx->topk_segs, ctx->d_topk_part, ctx->d_topk_ticket, d_topk_idx, no_noise, 1.f));
-  return TR_OK;
-}
-
-// ---------------------------------------------------------------------------------------------------
-// tr_topk_noalloc: the same kernel with its scratch in a fixed device array instead of context memory.
-//
-// Some callers of this library cannot allocate device memory at all: a plug-in running inside a serving
-// process that has handed every byte of HBM to its own pool (cudaMalloc simply fails there), or code on a
-// latency-critical path where the implicit device-wide synchronisation of cudaMalloc / cudaFree is not
-// acceptable.  tr_init allocates, so such callers cannot even create a context.  For them the per-segment
-// candidate lists and the per-row tickets of the top-k kernel live in the file-scope array below, which every
-// device that loads this library carries until the process exits.
-constexpr int NOALLOC_MAX_ROWS = 4096;            // logits rows per call
-constexpr int NOALLOC_MAX_PART = 65536;           // rows * segments * k partial keys per call
-constexpr size_t NOALLOC_TICKET_BYTES = sizeof(unsigned int) * NOALLOC_MAX_ROWS;
-constexpr size_t NOALLOC_BYTES = NOALLOC_TICKET_BYTES + sizeof(u64) * NOALLOC_MAX_PART;  // 528 KB
-
-static __device__ __align__(256) unsigned char g_noalloc_scratch[NOALLOC_BYTES];
-
-#include <mutex>
-namespace {
-constexpr int NOALLOC_MAX_DEVICES = 64;
-std::mutex g_noalloc_mutex;
-unsigned char* g_noalloc_ptr[NOALLOC_MAX_DEVICES] = {};  // device address of the array, per device
-}  // namespace
-
-extern "C" tr_status tr_topk_noalloc_limits(int32_t* max_rows, int32_t* max_partial_keys) {
-  if (!max_rows || !max_partial_keys) return TR_ERR_INVALID_ARG;
-  *max_rows = NOALLOC_MAX_ROWS;
-  *max_partial_keys = NOALLOC_MAX_PART;
-  return TR_OK;
-}
-
-extern "C" tr_status tr_topk_noalloc(const float* d_logits, int32_t rows, int32_t vocab, int32_t k,
-                                     int32_t* d_topk_idx, void* stream) {
-  if (!d_logits || !d_topk_idx || rows < 1 || k < 1 || k > TR_MAX_K || vocab < k) return TR_ERR_INVALID_ARG;
-  const int segs = (vocab + TOPK_SEG_ELEMS - 1) / TOPK_SEG_ELEMS;
-  if (rows > NOALLOC_MAX_ROWS || static_cast<int64_t>(rows) * segs * k > NOALLOC_MAX_PART || rows > 65535)
-    return TR_ERR_UNSUPPORTED;  // beyond the fixed scratch: see tr_topk_noalloc_limits
-  int dev = -1;
-  TR_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return TR_ERR_UNSUPPORTED;
-  unsigned char* base = nullptr;
-  {
-    // First call on this device: look up where this device keeps its copy of the array.  In host code the
-    // array's name is only a handle; the kernel must be given the address the runtime reports for it.
-    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
-    if (!g_noalloc_ptr[dev]) {
-      void* p = nullptr;
-      TR_CUDA_TRY(cudaGetSymbolAddress(&p, g_noalloc_scratch));
-      g_noalloc_ptr[dev] = static_cast<unsigned char*>(p);
-    }
-    base = g_noalloc_ptr[dev];
-  }
-  cudaStream_t s = static_cast<cudaStream_t>(stream);
-  unsigned int* ticket = reinterpret_cast<unsigned int*>(base);
-  u64* part = reinterpret_cast<u64*>(base + NOALLOC_TICKET_BYTES);
-  // The array keeps whatever the previous call left behind.  The tickets must start at zero; the partial lists
-  // are fully rewritten by every call before they are read.
-  TR_CUDA_TRY(cudaMemsetAsync(ticket, 0, sizeof(unsigned int) * rows, s));
-  const dim3 grid(segs, rows);
-  const bool vec = (vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
-  if (vec)
-    tr_topk_kernel<true, false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx, nullptr, 1.f);
-  else
-    tr_topk_kernel<false, false><<<grid, TOPK_THREADS, 0, s>>>(d_logits, vocab, k, segs, part, ticket, d_topk_idx, nullptr, 1.f);
-  TR_CUDA_TRY(cudaGetLastError());
+    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f)
+            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f);
+  TR_CUDA_TRY(e);
   return TR_OK;
 }

@@ -58,8 +58,6 @@ static tr_status free_all(tr_ctx* c) {
   cudaFree(c->d_level_off);
   cudaFree(c->d_anc);
   cudaFree(c->d_M);
-  cudaFree(c->d_topk_part);
-  cudaFree(c->d_topk_ticket);
   cudaFree(c->d_seq_ticket);
   cudaFree(c->d_lm_part);
   cudaFree(c->d_sampled);
@@ -83,6 +81,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   *out = nullptr;
   if (k < 1 || k > TR_MAX_K || vocab < k || batch < 1 || device < 0) return TR_ERR_INVALID_ARG;
   if (n_nodes < 1 || n_nodes > TR_MAX_NODES) return TR_ERR_TEMPLATE;
+  if (static_cast<int64_t>(batch) * n_nodes > 65535) return TR_ERR_UNSUPPORTED;  // logits rows are a grid's y extent
   // Template checks: layer order, parents before children, siblings contiguous enough for Algorithm 1.
   if (parent[0] != -1) return TR_ERR_TEMPLATE;
   std::vector<int32_t> depth(n_nodes, 0);
@@ -143,11 +142,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaMalloc(&c->d_M, m_bytes));
   TR_INIT_TRY(cudaMemset(c->d_M, 0, m_bytes));
 
-  c->topk_segs = (vocab + TOPK_SEG_ELEMS - 1) / TOPK_SEG_ELEMS;
   const size_t rows = static_cast<size_t>(batch) * n_nodes;
-  TR_INIT_TRY(cudaMalloc(&c->d_topk_part, sizeof(unsigned long long) * rows * c->topk_segs * k));
-  TR_INIT_TRY(cudaMalloc(&c->d_topk_ticket, sizeof(unsigned int) * rows));
-  TR_INIT_TRY(cudaMemset(c->d_topk_ticket, 0, sizeof(unsigned int) * rows));
   TR_INIT_TRY(cudaMalloc(&c->d_seq_ticket, sizeof(unsigned int) * batch));
   TR_INIT_TRY(cudaMemset(c->d_seq_ticket, 0, sizeof(unsigned int) * batch));
   TR_INIT_TRY(cudaMalloc(&c->d_sampled, sizeof(int32_t) * rows));
@@ -174,8 +169,6 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
     tr_status st = tr_attention_mma_setup();
     if (st == TR_OK) st = tr_attention_tc_setup();
     if (st == TR_OK) st = tr_lm_head_setup();
-    const char* force = getenv("TR_ATTN_FORCE_MMA");
-    c->force_mma = force && force[0] == '1';
     if (st != TR_OK) {
       free_all(c);
       return st;
@@ -193,7 +186,7 @@ extern "C" tr_status tr_destroy(tr_ctx* ctx) {
 }
 
 extern "C" tr_status tr_set_update_rule(tr_ctx* ctx, int32_t rule, int32_t scope) {
-  if (!ctx || (rule != TR_UPDATE_LAST && rule != TR_UPDATE_FIRST) ||
+  if (!ctx || (rule != TR_UPDATE_LAST && rule != TR_UPDATE_FIRST && rule != TR_UPDATE_CUR) ||
       (scope != TR_UPDATE_ALL_DRAFT && scope != TR_UPDATE_ONLY_ACCEPTED))
     return TR_ERR_INVALID_ARG;
   ctx->update_rule = rule;
@@ -207,6 +200,28 @@ extern "C" tr_status tr_matrix_zero(tr_ctx* ctx, void* stream) {
   if (!ctx) return TR_ERR_INVALID_ARG;
   const size_t bytes = sizeof(int32_t) * static_cast<size_t>(ctx->batch) * ctx->vocab * ctx->k;
   TR_CUDA_TRY(cudaMemsetAsync(ctx->d_M, 0, bytes, static_cast<cudaStream_t>(stream)));
+  return TR_OK;
+}
+
+// Seeded fill (Sec. 5.2 initialisation study, "Random"): every entry is a counter-based hash of its position.
+__global__ void tr_matrix_fill_kernel(int32_t* __restrict__ M, size_t n, int V, uint64_t seed) {
+  for (size_t i = blockIdx.x * static_cast<size_t>(blockDim.x) + threadIdx.x; i < n;
+       i += static_cast<size_t>(gridDim.x) * blockDim.x) {
+    uint64_t z = seed + 0x9E3779B97F4A7C15ull * (static_cast<uint64_t>(i) + 1ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    M[i] = static_cast<int32_t>(((z >> 32) * static_cast<uint64_t>(V)) >> 32);
+  }
+}
+
+extern "C" tr_status tr_matrix_fill(tr_ctx* ctx, int32_t mode, uint64_t seed, void* stream) {
+  if (!ctx || (mode != TR_FILL_ZERO && mode != TR_FILL_SEEDED)) return TR_ERR_INVALID_ARG;
+  if (mode == TR_FILL_ZERO) return tr_matrix_zero(ctx, stream);
+  const size_t n = static_cast<size_t>(ctx->batch) * ctx->vocab * ctx->k;
+  const int blocks = static_cast<int>(n / 256 + 1 < 1184 ? n / 256 + 1 : 1184);
+  tr_matrix_fill_kernel<<<blocks, 256, 0, static_cast<cudaStream_t>(stream)>>>(ctx->d_M, n, ctx->vocab, seed);
+  TR_CUDA_TRY(cudaGetLastError());
   return TR_OK;
 }
 
@@ -235,6 +250,7 @@ extern "C" tr_status tr_matrix_export(tr_ctx* ctx, int32_t seq, int32_t* host_M)
 
 extern "C" tr_status tr_device_flags(tr_ctx* ctx, uint32_t* host_flags) {
   if (!ctx || !host_flags) return TR_ERR_INVALID_ARG;
+  TR_CUDA_TRY(cudaSetDevice(ctx->device));
   TR_CUDA_TRY(cudaDeviceSynchronize());
   TR_CUDA_TRY(cudaMemcpy(host_flags, ctx->d_flags, sizeof(uint32_t), cudaMemcpyDeviceToHost));
   return TR_OK;
@@ -254,7 +270,7 @@ extern "C" tr_status tr_verify_update(tr_ctx* ctx, const float* d_logits, const 
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s);
   if (st != TR_OK) return st;
-  return tr_launch_tail(ctx, d_tree, out, s);
+  return tr_launch_tail(ctx, d_tree, out, s, nullptr, true);
 }
 
 extern "C" tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits, const float* d_gumbel,
@@ -274,7 +290,7 @@ extern "C" tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits
   // kernels are ordered on the stream)
   st = tr_launch_topk(ctx, d_logits, drawn, s, d_gumbel, inv_temperature, 1);
   if (st != TR_OK) return st;
-  return tr_launch_tail(ctx, d_tree, out, s, drawn);
+  return tr_launch_tail(ctx, d_tree, out, s, drawn, true);
 }
 
 extern "C" tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, void* stream) {
@@ -322,7 +338,7 @@ extern "C" tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* a, void*
   tr_status st = check_attn_args(ctx, a);
   if (st != TR_OK) return st;
   // head_dim 128 runs on the tcgen05 / TMA kernel; head_dim 64 on the warp-level MMA kernel
-  if (a->head_dim == 128 && !ctx->force_mma) return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
+  if (a->head_dim == 128) return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
   return tr_launch_attention_mma(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
@@ -350,6 +366,7 @@ extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_s
   if (!d_out || !io || !io->h_q || !io->h_tree_k || !io->h_tree_v || !io->h_logits || !io->h_ctx_len ||
       !io->d_logits_staging || !io->d_tree || !io->h_out || !io->h_n_new || !io->h_out_tokens || !io->h_next_tree)
     return TR_ERR_INVALID_ARG;
+  TR_CUDA_TRY(cudaSetDevice(ctx->device));
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   const int B = ctx->batch, N = ctx->n_nodes, L = a->n_layers, D = a->head_dim;
   const size_t esz = sizeof(__nv_bfloat16);
@@ -369,6 +386,9 @@ extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_s
   TR_CUDA_TRY(cudaEventRecord(ctx->ev_start, s));  // whatever the caller queued before comes first on all three
   TR_CUDA_TRY(cudaStreamWaitEvent(ctx->io_in, ctx->ev_start, 0));
   TR_CUDA_TRY(cudaStreamWaitEvent(ctx->io_out, ctx->ev_start, 0));
+  // the prefix lengths the kernels read on the device are this call's host values (the tree rows are placed by them)
+  TR_CUDA_TRY(cudaMemcpyAsync(const_cast<int32_t*>(a->d_ctx_len), io->h_ctx_len, sizeof(int32_t) * B,
+                              cudaMemcpyHostToDevice, ctx->io_in));
   const size_t q_layer = static_cast<size_t>(N) * a->n_q_heads * D;  // elements of one (sequence, layer) of Q / out
   for (int g = 0; g < G; ++g) {
     const int l0 = static_cast<int>(static_cast<int64_t>(L) * g / G), l1 = static_cast<int>(static_cast<int64_t>(L) * (g + 1) / G);
@@ -429,13 +449,5 @@ extern "C" tr_status tr_step_host(tr_ctx* ctx, const tr_attn_args* a, const tr_s
   TR_CUDA_TRY(cudaEventRecord(ctx->ev_out, ctx->io_out));
   TR_CUDA_TRY(cudaStreamWaitEvent(s, ctx->ev_out, 0));  // the caller's stream ends after the last copy out
   TR_CUDA_TRY(cudaStreamSynchronize(s));
-  return TR_OK;
-}
-
-// Debugging aid (not part of the public header): copies the first n floats of the split-KV scratch to the host.
-extern "C" tr_status tr_debug_read_scratch(tr_ctx* ctx, float* host, int32_t n) {
-  if (!ctx || !host || n < 0) return TR_ERR_INVALID_ARG;
-  TR_CUDA_TRY(cudaDeviceSynchronize());
-  TR_CUDA_TRY(cudaMemcpy(host, ctx->d_attn_part_o, sizeof(float) * n, cudaMemcpyDeviceToHost));
   return TR_OK;
 }

@@ -18,7 +18,7 @@
 
 void tr_set_last_cuda_error(cudaError_t e, const char* what, const char* file, int line);
 
-// Top-k of one logits row is computed by TOPK_SEG_ELEMS-wide segments, one CTA each.
+// The top-k kernels scan a logits row in pieces of TOPK_SEG_ELEMS values: 16 per thread of a 256-thread CTA.
 constexpr int TOPK_THREADS = 256;
 constexpr int TOPK_ELEMS_PER_THREAD = 16;
 constexpr int TOPK_SEG_ELEMS = TOPK_THREADS * TOPK_ELEMS_PER_THREAD;  // 4096
@@ -45,10 +45,7 @@ struct tr_ctx {
   uint32_t* d_anc = nullptr;     // [N][4] bit j of row i: j is i or an ancestor of i
   int32_t* d_M = nullptr;        // [batch][V][k]
   // scratch
-  unsigned long long* d_topk_part = nullptr;  // [batch*N][segs][k] packed (value, index) keys
-  unsigned int* d_topk_ticket = nullptr;      // [batch*N]
   unsigned int* d_seq_ticket = nullptr;       // [batch]: CTAs of a sequence that passed tr_commit's read phase
-  int topk_segs = 0;
   int32_t* d_sampled = nullptr;               // [batch*N] tokens drawn by tr_verify_update_sampled
   unsigned long long* d_lm_part = nullptr;    // [batch*N][lm_parts_cap][k] per-CTA lists of tr_lm_head_topk
   int lm_parts_cap = 0;
@@ -60,7 +57,6 @@ struct tr_ctx {
   cudaEvent_t ev_start = nullptr, ev_logits = nullptr, ev_out = nullptr;
   cudaEvent_t ev_in[TR_IO_GROUPS] = {}, ev_attn[TR_IO_GROUPS] = {};
   int update_rule = 0, update_scope = 0;  // TR_UPDATE_*
-  bool force_mma = false;  // debugging aid: TR_ATTN_FORCE_MMA=1 at tr_init keeps head_dim 128 on the warp-MMA kernel
 };
 
 // Launch with programmatic dependent launch: the kernel may be scheduled while the previous kernel of the stream is
@@ -90,8 +86,9 @@ __device__ __forceinline__ void tr_grid_dependency_wait() { asm volatile("gridde
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
                          const float* d_gumbel = nullptr, float inv_temperature = 1.f, int k_override = 0);
 // d_target [batch, N] (optional): the token every node's children are matched against, instead of topk[:, 0]
+// tree_early: d_tree was written at least two kernels back on the stream (the kernel directly in front did not write it)
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s,
-                         const int32_t* d_target = nullptr);
+                         const int32_t* d_target = nullptr, bool tree_early = false);
 tr_status tr_launch_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,
                            const int32_t* d_out_tokens, const int32_t* d_n_new, cudaStream_t s);
 tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);

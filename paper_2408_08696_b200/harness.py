@@ -15,6 +15,16 @@ def bf16_tensor(bits_u16, device):
     return torch.from_numpy(np.ascontiguousarray(bits_u16).view(np.int16)).to(device).view(torch.bfloat16)
 
 
+L2_BYTES = 126 << 20
+
+
+def rotation_larger_than_l2(w: synth.Workload, factor=1.5):
+    """Number of rotating logits buffers whose total size exceeds `factor` x the L2 capacity, so that in a loop that
+    cycles through them every step's logits come from HBM, not from a warm L2 (at least 4)."""
+    per_step = w.batch * w.n_nodes * w.vocab * 4
+    return max(4, -(-int(factor * L2_BYTES) // per_step))
+
+
 class DeviceWorkload:
     def __init__(self, w: synth.Workload, n_layers=None, device=0, n_rot=4, with_attention=True, splits=0,
                  zero_matrix=False):
@@ -67,27 +77,43 @@ class DeviceWorkload:
 
     def capture_graphs(self):
         """One CUDA graph per rotating logits buffer; replay graphs[i % n_rot] for step i = 0, 1, 2, ... in order.
-        Graph r holds the step's own kernels - attention, top-k, accept/update/retrieve - followed by the toy
-        model's patch of buffer r+1 for the NEXT step (the harness work sits at the end of the chain instead of
-        in front of the attention launch); buffer 0 is patched here, eagerly, for the first replay."""
+        Graph r holds the step's own kernels in a chain - attention, top-k, accept/update/retrieve - and, on a side
+        branch that joins the chain in front of the top-k kernel, the toy model's patch of buffer r for the tree
+        the previous step left (harness work: it stands for the rest of the model's forward pass, which produces
+        the logits while the step's attention runs)."""
         graphs = []
         s = torch.cuda.Stream(self.dev)
-        self.patch(0)
+        side = torch.cuda.Stream(self.dev)
         torch.cuda.synchronize(self.dev)
         with torch.cuda.stream(s):
             for r in range(self.n_rot):
                 g = torch.cuda.CUDAGraph()
                 with torch.cuda.graph(g, stream=s):
                     if self.attn is not None:
+                        side.wait_stream(s)
+                        self.patch(r, side)
                         tr.tr_tree_attention(self.ctx, self.attn, s)
+                        s.wait_stream(side)
+                    else:
+                        self.patch(r, s)
                     tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, s)
-                    self.patch((r + 1) % self.n_rot, s)
                 graphs.append(g)
         torch.cuda.synchronize(self.dev)
         return graphs
 
+    def reset(self):
+        """Back to the state right after construction (matrices, first tree, un-patched logits), so that a loop can
+        be run again from step 0 - for instance to check replayed graphs against the CPU checker."""
+        torch.cuda.synchronize(self.dev)
+        for b in range(self.w.batch):
+            tr.tr_matrix_import(self.ctx, b, self.M0[b])
+        self.d_logits.copy_(self.d_noise)
+        self.d_prev_col.fill_(-1)
+        tr.tr_build_tree(self.ctx, self.d_root, self.d_tree)
+        torch.cuda.synchronize(self.dev)
+
     def kernels_per_step(self):
-        n = 3  # logits patch (harness), top-k, accept/update/retrieve
+        n = 3  # logits patch (harness), top-k (one cluster per row), accept/update/retrieve
         if self.attn is not None:
             n += 1
             base = self.w.batch * self.L * self.w.n_q_heads

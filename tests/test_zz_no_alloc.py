@@ -1,10 +1,13 @@
 """The allocation-free top-k entry point, for callers that cannot call cudaMalloc (a process whose memory pool
 owns the whole device, or a loop that cannot take cudaMalloc's device-wide synchronisation).  It must give
-exactly what the context-based path gives, on two calls in a row (the scratch array is shared and keeps the
-previous call's contents).  Collected last on purpose: a failure here cannot hide other tests' results."""
+exactly what the context-based path gives - and what the CPU oracle's argtopk gives - on calls in a row (the scratch
+array is shared and keeps the previous call's contents).  Collected last on purpose: a failure here cannot hide
+other tests' results."""
 import numpy as np
 import pytest
 import torch
+
+from oracle import tr_oracle as orc
 
 pytestmark = pytest.mark.gpu
 
@@ -42,6 +45,7 @@ def test_no_alloc_topk_matches_context_path_twice_in_a_row():
     torch.cuda.synchronize()
     for (d_x, d_out), exp in zip(outs, expected):
         assert (d_out.cpu().numpy() == exp).all()                          # integer indices: bit-exact
+        assert (d_out.cpu().numpy() == orc.argtopk(d_x.cpu().numpy(), k)).all()
 
 
 def test_no_alloc_rejects_sizes_beyond_the_fixed_scratch():
