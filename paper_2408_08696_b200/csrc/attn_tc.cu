@@ -32,6 +32,9 @@ constexpr int WARP_PRODUCER = 8, WARP_MMA = 9, WARP_PV = 10;
 // Registers are re-balanced per warpgroup after start-up (setmaxnreg): 12 warps are launched at 168 each.
 constexpr int REGS_EPILOGUE = 112, REGS_SOFTMAX = 240, REGS_CONTROL = 96;
 
+TR_STAMP_DECL(g_attn_stamps, 8)
+TR_STAMP_DECL(g_attn_cta, 512)
+
 struct TcParams {
   __nv_bfloat16* out;
   const int32_t* ctx_len;
@@ -173,6 +176,11 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   auto bar = [&](int i) { return bars + static_cast<uint32_t>(i) * 8u; };
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+#ifdef TR_STAMPS
+  if (threadIdx.x == 0 && blockIdx.x == 0) g_attn_stamps[5] = g_attn_stamps[0];  // the previous launch's start
+#endif
+  TR_STAMP_MIN(g_attn_stamps, 0);
+  TR_STAMP_MAX(g_attn_stamps, 1);
   int* s_ctx = reinterpret_cast<int*>(base_ptr + SM_CTX);
   auto stage_ctx_len = [&]() {
     const int nb = p.n_units / (p.L * p.HU * p.S * p.MT);  // sequences
@@ -211,6 +219,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem = *s_tmem;
+  TR_STAMP_MAX(g_attn_stamps, 2);
   float* s_lm = reinterpret_cast<float*>(base_ptr + SM_LM);  // [2 O buffers][l: 128 | m: 128]
 
   // Each warpgroup first re-sizes its register budget: the light roles hand registers to the softmax warps.
@@ -536,6 +545,16 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
   // ---- teardown: every thread arrives here, also after an aborted wait
   __syncthreads();
+  TR_STAMP_MIN(g_attn_stamps, 3);
+  TR_STAMP_MAX(g_attn_stamps, 4);
+#ifdef TR_STAMPS
+  if (threadIdx.x == 0 && blockIdx.x < 256) {
+    unsigned smid;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+    g_attn_cta[blockIdx.x] = tr_globaltimer();
+    g_attn_cta[256 + blockIdx.x] = smid;
+  }
+#endif
   if (*s_abort) {
     if (tid == 0) atomicOr(p.flags, TR_FLAG_WAIT_TIMEOUT);
     // give copies and MMAs that may still be in flight time to land before shared memory and TMEM are released
@@ -604,6 +623,23 @@ __global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams 
 
 }  // namespace
 
+#ifdef TR_STAMPS
+extern "C" int tr_debug_stamps_attn_cta(unsigned long long* host) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host, g_attn_cta, sizeof(unsigned long long) * 512);
+  return 0;
+}
+extern "C" int tr_debug_stamps_attn(unsigned long long* host, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host, g_attn_stamps, sizeof(unsigned long long) * 8);
+  if (reset) {
+    unsigned long long init[8] = {~0ull, 0, 0, ~0ull, 0, 0, 0, 0};
+    cudaMemcpyToSymbol(g_attn_stamps, init, sizeof(init));
+  }
+  return 0;
+}
+#endif
+
 tr_status tr_attention_tc_setup() {
   TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
   TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
@@ -670,7 +706,11 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   // ring slot; otherwise Q is double-buffered so that short units overlap their Q load.
   if (p.MT > 1)
     tr_attn_tc_kernel<true, false><<<grid, NTHREADS, SMEM_BYTES, s>>>(mq, mk, mv, p);
+#ifdef TR_ATTN_PDL_ALWAYS
+  else if (true)
+#else
   else if (p.S > 1)
+#endif
     // a short launch (fewer units than SMs, split along the keys) between other short kernels, typically one layer's
     // attention: programmatic dependent launch hides its launch latency (503 -> 475 us for 32 per-layer launches at
     // the 7B shape).  Long launches gain nothing from it and measured about 1.5 % slower.

@@ -4,15 +4,19 @@
 // whose unsigned order IS that order, so all keys are distinct and "top-k" means "the k largest keys" - any split /
 // merge order gives the same answer, bit for bit.
 //
-// One thread-block cluster per logits row, P = 1, 2, 4 or 8 CTAs; CTA p scans a contiguous part of the row in chunks
-// of 4096 values (16 per thread in registers, 128-bit streaming loads).  The hot loop works on the float values only:
-//   threshold : tau = k-th largest of the chunk's 16 half-warp maxima (at least k values of the part are >= tau, so
-//               the part's k best keys are among the values >= tau); tau only grows from chunk to chunk
+// One thread-block cluster per logits row, P = 1, 2, 4 or 8 CTAs of 128 threads; CTA p scans a contiguous part of the
+// row in chunks of 4096 values (32 per thread in registers, 128-bit streaming loads).  The kernel is short and all its
+// CTAs are resident at once, so its duration is the memory latency plus the instructions every warp issues: the hot
+// loop works on the float values only and keeps the per-warp instruction count low.
+//   threshold : tau = k-th largest of the chunk's 16 quarter-warp maxima (at least k values of the part are >= tau,
+//               so the part's k best keys are among the values >= tau); tau only grows from chunk to chunk
 //   candidates: the few values >= tau are turned into keys and pushed to shared memory (threads whose own maximum is
-//               below tau skip the scan)
-//   part list : candidates ranked by counting -> the part's k best keys, stored straight into the shared memory of
-//               the cluster's first CTA (distributed shared memory)
-//   merge     : after one cluster barrier the first CTA ranks the P * k keys by counting and writes the row's top-k.
+//               below tau skip the scan; the others test four values at a time)
+//   part list : candidates ranked by counting (four threads per candidate) -> the part's k best keys, stored straight
+//               into the shared memory of EVERY CTA of the cluster (distributed shared memory)
+//   merge     : after one cluster barrier every CTA holds all P lists and ranks its own k keys among them by counting
+//               (eight threads per key); a key with fewer than k keys above it is written to its place of the row's
+//               top-k.  Keys are distinct, so the P CTAs write disjoint places.
 // No global scratch, no atomics on global memory, no second kernel.  Massive ties (more candidates than the buffer
 // holds) take an exact, slower path that selects round by round from global memory.
 #include "tr_internal.cuh"
@@ -20,10 +24,12 @@
 namespace {
 
 typedef unsigned long long u64;
-constexpr int CHUNK = TOPK_SEG_ELEMS;        // values per CTA and iteration
-constexpr int E = TOPK_ELEMS_PER_THREAD;     // values per thread and iteration
-constexpr int CAND_CAP = 512;
+constexpr int KT = 128;                      // threads per CTA
+constexpr int E = 32;                        // values per thread and iteration
+constexpr int CHUNK = KT * E;                // values per CTA and iteration (4096)
+constexpr int CAND_CAP = 512;                // candidate keys a CTA can hold
 constexpr int MAX_PARTS = 8;
+TR_STAMP_DECL(g_stamps, 16)
 
 // float -> uint32 whose unsigned order is the float order (-0 and +0 coincide), and back
 __device__ __forceinline__ uint32_t ord_u32(float v) {
@@ -48,25 +54,29 @@ __device__ __forceinline__ float max3f(float a, float b, float c) {
   asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
   return d;
 }
-// store into the shared memory of the cluster's CTA 0 (same offset as the local address `p`)
-__device__ __forceinline__ void st_leader_u64(const void* p, u64 v) {
+// store into the shared memory of every CTA of the cluster (same offset as the local address `p`)
+__device__ __forceinline__ void st_all_u64(const void* p, u64 v, int n_ctas) {
   const uint32_t local = static_cast<uint32_t>(__cvta_generic_to_shared(p));
-  uint32_t remote;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(0u));
-  asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+  for (int r = 0; r < n_ctas; ++r) {
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local), "r"(r));
+    asm volatile("st.shared::cluster.u64 [%0], %1;" ::"r"(remote), "l"(v) : "memory");
+  }
 }
+__device__ __forceinline__ int count_gt(const ulonglong2& a, u64 x) { return (a.x > x) + (a.y > x); }
 
 // kSample: rank z = fl32(fl32(logit * inv_t) + gumbel) instead of the logits (Sec. 5.3 temperature sampling: with k = 1
 // the result is the token drawn at temperature 1 / inv_t by the Gumbel-max rule).  Two roundings, no fused multiply-add:
 // the decision is reproducible with plain float32 arithmetic.
 template <bool kVec, bool kSample>
-__global__ void __launch_bounds__(TOPK_THREADS)
+__global__ void __launch_bounds__(KT)
 tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_part, int32_t* __restrict__ topk_idx,
                const float* __restrict__ gumbel, float inv_t) {
-  __shared__ u64 s_cand[CAND_CAP];
-  __shared__ u64 s_all[MAX_PARTS * TR_MAX_K];  // CTA 0 of the cluster: every part's list
-  __shared__ u64 s_red[TOPK_THREADS / 32];
-  __shared__ uint32_t s_gmax[2][16];
+  __shared__ __align__(16) u64 s_cand[CAND_CAP + 32];        // candidates, then up to 32 zeros of padding
+  __shared__ __align__(16) u64 s_all[MAX_PARTS * TR_MAX_K];  // every part's list (each CTA gets a copy)
+  __shared__ u64 s_red[KT / 32];
+  __shared__ uint32_t s_gmax[16];
+  __shared__ uint32_t s_tau;
   __shared__ int s_cnt;
 
   const int part = blockIdx.x, P = gridDim.x, row = blockIdx.y;
@@ -76,25 +86,29 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
   const int part_base = part * chunks_per_part * CHUNK;
   const int part_end = min(V, part_base + chunks_per_part * CHUNK);
 
-  if (tid == 0) s_cnt = 0;
-  // first half of a cluster barrier: before a CTA stores into the first CTA's shared memory (below), every CTA of the
+  TR_STAMP_MIN(g_stamps, 0);
+  if (tid == 0) { s_tau = 0u; s_cnt = 0; }  // tau = 0 is below every value, -inf included
+  // first half of a cluster barrier: before a CTA stores into another CTA's shared memory (below), every CTA of the
   // cluster must have started
   if (P > 1) asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
   // (programmatic dependent launch) the logits belong to whatever ran before on this stream
   tr_grid_dependency_wait();
+  TR_STAMP_MIN(g_stamps, 1);
+  TR_STAMP_MAX(g_stamps, 2);
   // The kernel behind this one (accept / update / retrieve) may be scheduled from here on and run its preamble; it
   // waits for this grid to finish before it reads the result.  (Only after the wait above: whatever that kernel
   // fetches early must come from kernels that are complete by now.)
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // value j of this thread: vector layout - float4 number j/4 of the chunk's tid-th slot; scalar layout - strided
   auto index_of = [&](int base, int j) -> int {
-    return kVec ? base + (j >> 2) * (TOPK_THREADS * 4) + tid * 4 + (j & 3) : base + j * TOPK_THREADS + tid;
+    return kVec ? base + (j >> 2) * (KT * 4) + tid * 4 + (j & 3) : base + j * KT + tid;
   };
   auto load_chunk = [&](int base, float (&v)[E]) {
     if (kVec) {
 #pragma unroll
       for (int j = 0; j < E / 4; ++j) {
-        const int i0 = base + j * (TOPK_THREADS * 4) + tid * 4;
+        const int i0 = base + j * (KT * 4) + tid * 4;
         float4 t = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         if (i0 < part_end) {
           t = __ldcs(reinterpret_cast<const float4*>(rowp + i0));
@@ -109,7 +123,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
     } else {
 #pragma unroll
       for (int j = 0; j < E; ++j) {
-        const int i = base + j * TOPK_THREADS + tid;
+        const int i = base + j * KT + tid;
         float x = -INFINITY;
         if (i < part_end) {
           x = __ldcs(rowp + i);
@@ -121,50 +135,63 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
   };
 
   // ---- scan the part chunk by chunk; the next chunk's loads are in flight while the current one is examined
-  uint32_t tau_ord = 0u;  // below every value, -inf included
   float v[E], vn[E];
   if (part_base < part_end) load_chunk(part_base, v);
+  TR_STAMP_MIN(g_stamps, 6);
   for (int c = 0; c < chunks_per_part; ++c) {
     const int base = part_base + c * CHUNK;
     if (base >= part_end) break;  // uniform over the CTA
     const bool more = (c + 1 < chunks_per_part) && (base + CHUNK < part_end);
     if (more) load_chunk(base + CHUNK, vn);
-    // thread maximum (values only: -0 == +0, no NaN by precondition), then the maxima of the 16 half-warp groups
-    float m = max3f(v[0], v[1], v[2]);
+    // maxima of groups of four values and of the thread (values only: -0 == +0, no NaN by precondition), then the
+    // maxima of the 16 quarter-warp groups
+    float g4[E / 4];
 #pragma unroll
-    for (int j = 3; j + 1 < E; j += 2) m = max3f(m, v[j], v[j + 1]);
-    m = fmaxf(m, v[E - 1]);
+    for (int j = 0; j < E / 4; ++j) g4[j] = fmaxf(max3f(v[4 * j], v[4 * j + 1], v[4 * j + 2]), v[4 * j + 3]);
+    float m = max3f(g4[0], g4[1], g4[2]);
+#pragma unroll
+    for (int j = 3; j + 1 < E / 4; j += 2) m = max3f(m, g4[j], g4[j + 1]);
+    m = fmaxf(m, g4[E / 4 - 1]);
     {
-      const unsigned mask = (lane < 16) ? 0x0000FFFFu : 0xFFFF0000u;
-      const uint32_t gm = __reduce_max_sync(mask, ord_u32(m));
-      if ((lane & 15) == 0) s_gmax[c & 1][tid >> 4] = gm;
+      const uint32_t gm = __reduce_max_sync(0xFFu << (lane & 24), ord_u32(m));
+      if ((lane & 7) == 0) s_gmax[tid >> 3] = gm;
     }
     __syncthreads();
-    // every warp works the threshold out for itself: the group maximum with fewer than k larger and at least k
-    // larger-or-equal ones is the k-th largest.  Groups past the row's end hold -inf; with fewer than k real groups
-    // the threshold is -inf and every value of the chunk is a candidate.
-    {
-      const uint32_t mine = s_gmax[c & 1][lane & 15];
+    // the first warp works the threshold out: the group maximum with fewer than k larger and at least k
+    // larger-or-equal ones is the k-th largest (lane = (group, half): each lane counts over 8 of the 16 maxima).
+    // Groups past the row's end hold -inf; with fewer than k real groups the threshold is -inf and every value of the
+    // chunk is a candidate.
+    if (tid < 32) {
+      const uint32_t mine = s_gmax[lane & 15];
       int larger = 0, ge = 0;
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const uint32_t g = s_gmax[c & 1][i];
+      for (int u = 0; u < 8; ++u) {
+        const uint32_t g = s_gmax[(lane >> 4) * 8 + u];
         larger += (g > mine) ? 1 : 0;
         ge += (g >= mine) ? 1 : 0;
       }
+      larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 16);
+      ge += __shfl_xor_sync(0xFFFFFFFFu, ge, 16);
       const unsigned hit = __ballot_sync(0xFFFFFFFFu, larger < k && ge >= k);
       const uint32_t tau_c = hit ? __shfl_sync(0xFFFFFFFFu, mine, __ffs(hit) - 1) : 0u;  // k <= 16 groups: always a hit
-      tau_ord = max(tau_ord, tau_c);
+      if (lane == 0) s_tau = max(s_tau, tau_c);
     }
-    const float tau = ord_to_float(tau_ord);
-    if (m >= tau) {
+    __syncthreads();
+    const float tau = ord_to_float(s_tau);
+    TR_STAMP_MIN(g_stamps, 7);
+    if (m >= tau) {  // a few threads per warp
 #pragma unroll
-      for (int j = 0; j < E; ++j) {
-        if (v[j] >= tau) {
-          const int i = index_of(base, j);
-          if (i < part_end) {
-            const int p = atomicAdd(&s_cnt, 1);
-            if (p < CAND_CAP) s_cand[p] = topk_key(v[j], i);
+      for (int j = 0; j < E / 4; ++j) {
+        if (g4[j] >= tau) {
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            if (v[4 * j + u] >= tau) {
+              const int i = index_of(base, 4 * j + u);
+              if (i < part_end) {
+                const int pos = atomicAdd(&s_cnt, 1);
+                if (pos < CAND_CAP) s_cand[pos] = topk_key(v[4 * j + u], i);
+              }
+            }
           }
         }
       }
@@ -175,26 +202,43 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
     }
   }
   __syncthreads();
-
-  // ---- the part's k best keys -> list `part` in the first CTA's shared memory (unused entries are 0)
-  u64* my_list = s_all + part * TR_MAX_K;
   const int cnt = s_cnt;
+  if (cnt <= CAND_CAP && tid < 32) s_cand[cnt + tid] = 0ull;  // zeros (below every key) pad the last round of 32
+  __syncthreads();
+  TR_STAMP_MAX(g_stamps, 3);
+  TR_STAMP_MIN(g_stamps, 8);
+
+  // ---- the part's k best keys -> list `part` in every CTA's shared memory (unused entries are 0)
+  u64* my_list = s_all + part * TR_MAX_K;
   if (P > 1) asm volatile("barrier.cluster.wait.aligned;" ::: "memory");
   if (cnt <= CAND_CAP) {
-    for (int t = tid; t < cnt; t += TOPK_THREADS) {
-      const u64 mine = s_cand[t];
+    // rank by counting, four threads per candidate: thread (c, s) counts the keys above candidate c among the
+    // entries s, s + 4, s + 8, ... - eight independent loads per round of 32 entries
+    const int s4 = tid & 3;
+    for (int c0 = 0; c0 < cnt; c0 += KT / 4) {
+      const int c = c0 + (tid >> 2);
+      const u64 mine = c < cnt ? s_cand[c] : ~0ull;
       int larger = 0;
-      for (int i = 0; i < cnt; ++i) larger += (s_cand[i] > mine) ? 1 : 0;
-      if (larger < k) st_leader_u64(my_list + larger, mine);
+      for (int i0 = 0; i0 < cnt; i0 += 32) {
+        u64 e[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) e[u] = s_cand[i0 + s4 + 4 * u];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) larger += (e[u] > mine) ? 1 : 0;
+      }
+      larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 1);
+      larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 2);
+      if (s4 == 0 && c < cnt && larger < k) st_all_u64(my_list + larger, mine, P);
     }
-    if (tid >= cnt && tid < k) st_leader_u64(my_list + tid, 0ull);
+    // entries the part cannot fill, and the unused tail of the list, are 0
+    if (tid < TR_MAX_K && (tid >= k || tid >= cnt)) st_all_u64(my_list + tid, 0ull, P);
   } else {
     // More candidates than the buffer holds (massive ties or adversarial layouts): select straight from global
     // memory, round by round, the whole CTA taking part.
     u64 last = ~0ull;
     for (int r = 0; r < k; ++r) {
       u64 best = 0;
-      for (int i = part_base + tid; i < part_end; i += TOPK_THREADS) {
+      for (int i = part_base + tid; i < part_end; i += KT) {
         float x = __ldcg(rowp + i);
         if (kSample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcg(rowg + i));
         const u64 key = topk_key(x, i);
@@ -206,34 +250,61 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
       __syncthreads();
       u64 mx = 0;
 #pragma unroll
-      for (int w = 0; w < TOPK_THREADS / 32; ++w) mx = s_red[w] > mx ? s_red[w] : mx;
+      for (int w = 0; w < KT / 32; ++w) mx = s_red[w] > mx ? s_red[w] : mx;
       last = mx;
-      if (tid == 0) st_leader_u64(my_list + r, mx);
+      if (tid == 0) st_all_u64(my_list + r, mx, P);
     }
+    if (tid >= k && tid < TR_MAX_K) st_all_u64(my_list + tid, 0ull, P);
   }
 
-  // ---- merge in the cluster's first CTA
+  // ---- every CTA now ranks its own list's keys among all lists
+  TR_STAMP_MIN(g_stamps, 9);
   if (P > 1) {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    if (part != 0) return;  // the lists are delivered; only the first CTA goes on
+    TR_STAMP_MIN(g_stamps, 10);
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   } else {
     __syncthreads();
   }
-  const int n = P * TR_MAX_K;
-  if (tid < n && (tid & (TR_MAX_K - 1)) < k) {
-    const u64 mine = s_all[tid];
-    if (mine != 0ull) {
-      int larger = 0;
-      for (int q = 0; q < P; ++q)
-        for (int i = 0; i < k; ++i) larger += (s_all[q * TR_MAX_K + i] > mine) ? 1 : 0;
-      if (larger < k)
-        topk_idx[static_cast<size_t>(row) * k + larger] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(mine));
+  TR_STAMP_MIN(g_stamps, 11);
+  TR_STAMP_MAX(g_stamps, 4);
+  {
+    // eight threads per key: thread (i, q) counts the keys of list q above key i of this part's list
+    const int i = tid >> 3, q = tid & 7;
+    const u64 mine = my_list[i];
+    int larger = 0;
+    if (q < P) {
+      const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(s_all + q * TR_MAX_K);
+      const ulonglong2 a0 = lp[0], a1 = lp[1], a2 = lp[2], a3 = lp[3];
+      larger = count_gt(a0, mine) + count_gt(a1, mine) + count_gt(a2, mine) + count_gt(a3, mine);
+      if (k > 8) {
+        const ulonglong2 a4 = lp[4], a5 = lp[5], a6 = lp[6], a7 = lp[7];
+        larger += count_gt(a4, mine) + count_gt(a5, mine) + count_gt(a6, mine) + count_gt(a7, mine);
+      }
     }
+    larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 1);
+    larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 2);
+    larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 4);
+    if (q == 0 && mine != 0ull && larger < k)
+      topk_idx[static_cast<size_t>(row) * k + larger] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(mine));
   }
+  TR_STAMP_MAX(g_stamps, 5);
+  TR_STAMP_MIN(g_stamps, 12);
 }
 
 }  // namespace
+
+#ifdef TR_STAMPS
+extern "C" int tr_debug_stamps_topk(unsigned long long* host, int reset) {
+  cudaDeviceSynchronize();
+  cudaMemcpyFromSymbol(host, g_stamps, sizeof(unsigned long long) * 16);
+  if (reset) {
+    unsigned long long init[16] = {~0ull, ~0ull, 0, 0, 0, 0, 0, 0};
+    cudaMemcpyToSymbol(g_stamps, init, sizeof(init));
+  }
+  return 0;
+}
+#endif
 
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
                          const float* d_gumbel, float inv_temperature, int k_override) {
@@ -248,7 +319,7 @@ tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx
 
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(P, rows);
-  cfg.blockDim = dim3(TOPK_THREADS);
+  cfg.blockDim = dim3(KT);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = s;
   cudaLaunchAttribute attr[2];

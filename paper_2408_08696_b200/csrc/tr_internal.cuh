@@ -80,6 +80,26 @@ inline cudaError_t tr_launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block
 __device__ __forceinline__ void tr_grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 #endif
 
+// Timeline instrumentation for development builds (-DTR_STAMPS): each translation unit keeps a few %globaltimer
+// stamps (earliest / latest over its CTAs) that a debug entry point copies out.  Compiled out of the product build.
+#ifdef TR_STAMPS
+#define TR_STAMP_DECL(name, n) static __device__ unsigned long long name[n];
+#ifdef __CUDACC__
+__device__ __forceinline__ unsigned long long tr_globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// "MIN": the first CTA's time of the latest launch (plain store); "MAX": the latest time over all CTAs so far
+#define TR_STAMP_MIN(arr, i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) arr[i] = tr_globaltimer(); } while (0)
+#define TR_STAMP_MAX(arr, i) do { if (threadIdx.x == 0) atomicMax(&arr[i], tr_globaltimer()); } while (0)
+#endif
+#else
+#define TR_STAMP_DECL(name, n)
+#define TR_STAMP_MIN(arr, i) do { } while (0)
+#define TR_STAMP_MAX(arr, i) do { } while (0)
+#endif
+
 // launchers (host functions defined next to their kernels)
 // With d_gumbel: the kernel ranks z = fl32(fl32(logit * inv_temperature) + gumbel) instead of the logits, k_override
 // entries per row (1: the draw of temperature sampling).
