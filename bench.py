@@ -29,11 +29,18 @@ UNIT = "us/step"
 
 
 def load_peaks():
+    """(HBM GB/s, sustained dense bf16 TFLOP/s, where they come from)."""
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
         d = json.load(open(p))
-        return float(d["hbm_gbs"]), "measured (MEASURED_PEAKS.json, copy bandwidth)"
-    return 6650.0, "fallback (earlier measurement on this pool)"
+        return (float(d["hbm_gbs"]), float(d.get("bf16_tflops_sustained", 1400.0)),
+                "measured (MEASURED_PEAKS.json: copy bandwidth, sustained cuBLAS bf16)")
+    return 6650.0, 1400.0, "fallback (earlier measurement on this pool)"
+
+
+def attention_flops(w, n_layers):
+    """4 N Hq (C_b + N) D per sequence and layer: the two products over the prefix and the whole tree block."""
+    return sum(4 * w.n_nodes * w.n_q_heads * (c + w.n_nodes) * w.head_dim for c in w.ctx) * n_layers
 
 
 def algorithmic_bytes(w, n_layers):
@@ -47,43 +54,54 @@ def algorithmic_bytes(w, n_layers):
 
 
 class ClockSampler:
-    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
-              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    """nvidia-smi in query mode (read-only) every 25 ms; `stop(t0, t1)` keeps the samples taken between the two host
+    times, i.e. during the timed region."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+    BAD = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown")
 
     def __init__(self, index):
         self.proc = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(index), "--query-gpu=" + self.FIELDS, "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "25"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             pass
 
-    def stop(self):
+    def stop(self, t0, t1):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.06)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        import datetime
+        sm, mx, reasons, n_all = [], [], set(), 0
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
         for line in out.splitlines():
             f = [x.strip() for x in line.split(",")]
-            if len(f) < 6:
+            if len(f) < 7:
                 continue
             try:
-                sm.append(float(f[0])); mx.append(float(f[1]))
+                ts = datetime.datetime.strptime(f[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                clk, cmax = float(f[1]), float(f[2])
             except ValueError:
                 continue
-            for n, v in zip(names, f[2:6]):
+            n_all += 1
+            if ts < t0 - 0.03 or ts > t1 + 0.03:      # a sample describes the ~25 ms before its time stamp
+                continue
+            sm.append(clk); mx.append(cmax)
+            for n, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_min_mhz": min(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "samples_outside_region": n_all - len(sm),
+                "reasons": sorted(reasons), "sampled": "every 25 ms during the timed blocks"}
 
 
 # ---------------------------------------------------------------------------------------------------
@@ -187,9 +205,10 @@ def measure_lm_head(torch, tr, dw, w, dev, reps=20):
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) / reps * 1000.0
-    passes = (rows + 127) // 128                               # one pass over the weight per 128 rows
-    byts = passes * w.vocab * H * 2 + rows * H * 2 + rows * w.k * 4
+    passes = (rows + 127) // 128                               # the kernel streams the weight once per 128 rows
+    byts = w.vocab * H * 2 + rows * H * 2 + rows * w.k * 4      # algorithmic: the weight ONCE, hidden states, output
     return {"us": us, "bound": "hbm", "achieved": byts / us / 1e3, "unit": "GB/s", "algorithmic_bytes": byts,
+            "weight_passes": passes, "weight_bytes_streamed": passes * w.vocab * H * 2,
             "rows": rows, "hidden": H, "vocab": w.vocab, "gpu_launches": passes + 1,
             "device_flags": tr.tr_device_flags(dw.ctx)}
 
@@ -240,6 +259,49 @@ def measure_sampled_verify(torch, tr, dw, w, dev, reps=20):
             "device_flags": tr.tr_device_flags(dw.ctx)}
 
 
+def check_parity(torch, tr, harness, dw, w, graphs, round_graph):
+    """Outside the timed region: the very graphs that were timed, replayed from the initial state, against the CPU
+    oracle - every integer output of 4 single-step replays, then one whole-round replay (n_rot steps in one graph):
+    last step's integer outputs, the matrices, and a seeded sample of 8 attention heads."""
+    from oracle import tr_oracle as orc
+    from paper_2408_08696_b200 import synth
+    from tests.oracle_loop import OracleLoop, attention_close, compare_step
+    res = {"single_step_replays": 4, "round_replay_steps": dw.n_rot, "attention_heads": 8}
+    try:
+        dw.reset()
+        ol = OracleLoop(w, n_rot=dw.n_rot)
+        for i in range(4):
+            graphs[i].replay()
+            compare_step(ol.step(i), dw.snapshot(), dw.ctx.max_new)
+        dw.reset()
+        ol = OracleLoop(w, n_rot=dw.n_rot)
+        dw.o.zero_()
+        round_graph.replay()
+        recs = [ol.step(i) for i in range(dw.n_rot)][-1]
+        compare_step(recs, dw.snapshot(), dw.ctx.max_new)
+        for b in range(w.batch):
+            assert (tr.tr_matrix_export(dw.ctx, b) == ol.M[b]).all(), "matrix differs"
+        import dataclasses
+        pool = synth.normal_pool(w.seed)
+        rng = np.random.default_rng(99)
+        group = w.n_q_heads // w.n_kv_heads
+        ws = dataclasses.replace(w, n_layers=dw.L)                # the slices are cut for the layer count in use
+        worst = [0.0, 0.0]
+        for _ in range(8):
+            b, l, h = int(rng.integers(0, w.batch)), int(rng.integers(0, dw.L)), int(rng.integers(0, w.n_q_heads))
+            qs, ks, vs = synth.attention_slice(ws, pool, b, l, h // group)
+            ref = orc.tree_attention(synth.bf16_bits_to_f32(qs[:, h:h + 1]), synth.bf16_bits_to_f32(ks)[None],
+                                     synth.bf16_bits_to_f32(vs)[None], w.ctx[b], dw.parent)
+            mx, rel = attention_close(dw.o[b, l, :, h].float().cpu().numpy(), ref[:, 0])
+            assert mx <= 2e-2 and rel <= 1e-2, ("attention", b, l, h, mx, rel)
+            worst = [max(worst[0], mx), max(worst[1], rel)]
+        assert tr.tr_device_flags(dw.ctx) == 0
+        res.update(ok=True, attention_max_abs=worst[0], attention_rel_l2=worst[1])
+    except AssertionError as e:
+        res.update(ok=False, error=str(e)[:200])
+    return res
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
@@ -257,68 +319,90 @@ def run_ours(args, w):
         dist.init_process_group("nccl", device_id=dev)
     K, W = args.steps, max(args.warmup, 3)
 
-    dw = harness.DeviceWorkload(w, n_layers=args.layers or None, device=local_rank)
-    graphs = dw.capture_graphs()
+    # rotating logits buffers larger than L2 in total, so that every step's logits come from HBM like its K/V
+    n_rot = harness.rotation_larger_than_l2(w)
+    dw = harness.DeviceWorkload(w, n_layers=args.layers or None, device=local_rank, n_rot=n_rot)
+    graphs = dw.capture_graphs()          # one step per graph
+    round_graph = dw.capture_round()      # n_rot steps in one graph
+
+    def run_steps(n):
+        """n steps: whole rounds as one graph launch each, the rest as single-step graphs."""
+        q, r = divmod(n, n_rot)
+        for _ in range(q):
+            round_graph.replay()
+        for i in range(r):
+            graphs[i].replay()
+
     if args.profile:
-        for i in range(W + K):
-            graphs[i % dw.n_rot].replay()  # rotation order
+        run_steps(W + K)
         torch.cuda.synchronize()
         dw.close()
         return
     stream = torch.cuda.current_stream()
-    step_no = 0  # the graphs must be replayed in rotation order (each patches the next one's logits)
-    for _ in range(W):
-        graphs[step_no % dw.n_rot].replay()
-        step_no += 1
+    run_steps(W)
     torch.cuda.synchronize()
-
-    # ---- timed region: K graph replays back to back, device time between two events on the launching stream
-    replicas.barrier()
-    torch.cuda.synchronize()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    # a first estimate of the step time sizes the number of timed blocks
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record(stream)
-    for _ in range(K):
-        graphs[step_no % dw.n_rot].replay()
-        step_no += 1
+    run_steps(K)
     e1.record(stream)
     torch.cuda.synchronize()
-    replicas.barrier()
-    elapsed_ms = e0.elapsed_time(e1)
-    if sampler:
-        # the timed region lasts tens of milliseconds; keep the same load running (untimed) for about half a second
-        # so that nvidia-smi's 100 ms samples see the clocks under this load
-        t_end = time.perf_counter() + 0.6
-        while time.perf_counter() < t_end:
-            for _ in range(50):
-                graphs[step_no % dw.n_rot].replay()
-                step_no += 1
+    est_ms = max(e0.elapsed_time(e1), 1e-3)
+    n_blocks = int(min(400, max(5, np.ceil(args.min_timed_ms / est_ms))))
+    if world > 1:  # every rank must run the same number of blocks
+        t = torch.tensor([n_blocks], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        n_blocks = int(t.item())
+
+    # ---- timed region: n_blocks blocks of exactly K steps; each block is bracketed by a barrier and a device
+    #      synchronisation on both sides and timed on the device (two events on the launching stream); the clocks
+    #      are sampled while the blocks run.  value = median block (per block: slowest rank).
+    for attempt in range(2):
+        sampler = ClockSampler(local_rank) if rank == 0 else None
+        if sampler:
+            time.sleep(0.25)              # let nvidia-smi come up before the region starts
+        block_ms = []
+        t_begin = time.time()
+        for _ in range(n_blocks):
+            replicas.barrier()
             torch.cuda.synchronize()
-    clocks = sampler.stop() if sampler else None
-    agg = replicas.aggregate(elapsed_ms, K, device=dev if world > 1 else "cpu")
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            run_steps(K)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            replicas.barrier()
+            block_ms.append(e0.elapsed_time(e1))
+        t_end = time.time()
+        clocks = sampler.stop(t_begin, t_end) if sampler else None
+        if not clocks or not (set(clocks["reasons"]) & set(ClockSampler.BAD)):
+            break
+        clocks["note"] = "first attempt saw %s and was measured again" % clocks["reasons"]
+    block_ms = replicas.max_over_ranks_vec(block_ms, device=dev if world > 1 else "cpu")
+    med_ms = float(np.median(block_ms))
+    agg = replicas.aggregate(med_ms, K, device="cpu", reduce=False)
     flags = tr.tr_device_flags(dw.ctx)
     # acceptance statistic of the toy model (a sanity figure, not a result): 64 untimed steps, n_new read each step
     n_new_sum, n_stat = 0, 64
-    for _ in range(n_stat):
-        graphs[step_no % dw.n_rot].replay()
-        step_no += 1
+    for i in range(n_stat):
+        graphs[i % n_rot].replay()
         n_new_sum += int(dw.out["n_new"].sum().item())
 
     # ---- dominant kernel (tree attention) alone: event pair around every launch, same stream
+    time.sleep(0.3)
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
     for i in range(K):
-        tr.trs_patch_logits(dw.d_logits[i % dw.n_rot], dw.d_noise[i % dw.n_rot], dw.d_tree,
-                            dw.d_prev_col[i % dw.n_rot], dw.d_succ, w.boost)
+        r = i % n_rot
+        tr.trs_patch_logits(dw.d_logits[r], dw.d_noise[r], dw.d_tree, dw.d_prev_col[r], dw.d_succ, w.boost)
         ev[i][0].record(stream)
         tr.tr_tree_attention(dw.ctx, dw.attn)
         ev[i][1].record(stream)
-        tr.tr_verify_update(dw.ctx, dw.d_logits[i % dw.n_rot], dw.d_tree, dw.out_struct)
+        tr.tr_verify_update(dw.ctx, dw.d_logits[r], dw.d_tree, dw.out_struct)
     torch.cuda.synchronize()
     attn_ms = float(np.mean([a.elapsed_time(b) for a, b in ev]))
     # per-layer launches (one call per layer, as a real model's forward would issue them), for the record
     per_layer_ms = None
     if dw.L > 1:
-        qs = [dw.q[:, l:l + 1] for l in range(dw.L)]
         args_l = [tr.make_attn_args(dw.ctx, dw.q[:, l:l + 1], dw.k[:, l:l + 1], dw.v[:, l:l + 1], dw.o[:, l:l + 1],
                                     dw.d_ctx_len, w.max_ctx) for l in range(dw.L)]
         gl = torch.cuda.CUDAGraph()
@@ -343,7 +427,7 @@ def run_ours(args, w):
     h_q = dw.q.cpu().pin_memory()
     h_tk = torch.stack([dw.k[b, :, :, c:c + N] for b, c in enumerate(w.ctx)]).cpu().contiguous().pin_memory()
     h_tv = torch.stack([dw.v[b, :, :, c:c + N] for b, c in enumerate(w.ctx)]).cpu().contiguous().pin_memory()
-    h_logits = [dw.d_noise[r].cpu().pin_memory() for r in range(dw.n_rot)]
+    h_logits = [dw.d_noise[r].cpu().pin_memory() for r in range(min(4, n_rot))]
     h_ctx = np.array(w.ctx, dtype=np.int32)
     h_out = torch.zeros(B, L, N, Hq, D, dtype=torch.bfloat16).pin_memory()
     h_n_new = torch.zeros(B, dtype=torch.int32).pin_memory()
@@ -355,33 +439,45 @@ def run_ours(args, w):
     io.h_ctx_len, io.d_logits_staging, io.d_tree = h_ctx.ctypes.data, d_stage.data_ptr(), dw.d_tree.data_ptr()
     io.h_out, io.h_n_new, io.h_out_tokens, io.h_next_tree = (h_out.data_ptr(), h_n_new.data_ptr(), h_tok.data_ptr(),
                                                              h_next.data_ptr())
-    h2d = h_q.numel() * 2 + h_tk.numel() * 2 + h_tv.numel() * 2 + h_logits[0].numel() * 4
+    h2d = h_q.numel() * 2 + h_tk.numel() * 2 + h_tv.numel() * 2 + h_logits[0].numel() * 4 + h_ctx.nbytes
     d2h = h_out.numel() * 2 + h_n_new.numel() * 4 + h_tok.numel() * 4 + h_next.numel() * 4
     Ke = max(3, min(K, 20))
     for i in range(2):
-        io.h_logits = h_logits[i % dw.n_rot].data_ptr()
+        io.h_logits = h_logits[i % len(h_logits)].data_ptr()
         tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)
     replicas.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
     for i in range(Ke):
-        io.h_logits = h_logits[i % dw.n_rot].data_ptr()
+        io.h_logits = h_logits[i % len(h_logits)].data_ptr()
         tr.tr_step_host(dw.ctx, dw.attn, dw.out_struct, io)      # synchronises the stream itself
     e2e_ms = (time.perf_counter() - t0) * 1000.0
     e2e = replicas.aggregate(e2e_ms, Ke, device=dev if world > 1 else "cpu")
 
     lm = measure_lm_head(torch, tr, dw, w, dev) if rank == 0 else None
     sampled_verify = measure_sampled_verify(torch, tr, dw, w, dev) if rank == 0 else None
+    parity = check_parity(torch, tr, harness, dw, w, graphs, round_graph) if rank == 0 else None
 
     if rank == 0:
-        peak, peak_src = load_peaks()
+        hbm_peak, tf_peak, peak_src = load_peaks()
         ab = algorithmic_bytes(w, dw.L)
+        fl = attention_flops(w, dw.L)
         attn_gbs = ab["attention"] / (attn_ms * 1e-3) / 1e9
+        attn_tfs = fl / (attn_ms * 1e-3) / 1e12
         step_gbs = ab["total"] / (agg["ms_per_step"] * 1e-3) / 1e9
+        hbm = {"achieved": attn_gbs, "peak": hbm_peak, "unit": "GB/s", "frac": attn_gbs / hbm_peak}
+        tensor = {"achieved": attn_tfs, "peak": tf_peak, "unit": "TFLOP/s", "frac": attn_tfs / tf_peak,
+                  "flops_per_launch": fl, "peak_kind": "sustained dense bf16 (the launch runs inside a long step)"}
+        bound = "tensor" if tensor["frac"] > hbm["frac"] else "hbm"
+        top = tensor if bound == "tensor" else hbm
         smp = OracleSampler(w)
         cpu_units, cpu_steps = 2048, 3                       # roughly 15-20 s of host work at the 7B shape
         cpu_us = float(np.mean([smp.step_us(cpu_units) for _ in range(cpu_steps)]))
         cpu_desc, cpu_threads = smp.describe(cpu_units, cpu_steps), smp.threads
+        kv_mb = ab["attention"] / 1e6
+        l2_note = ("inputs larger than L2: %.0f MB of K/V and %d rotating logits buffers (%.0f MB) per round"
+                   % (kv_mb, n_rot, n_rot * ab["logits"] / 1e6)) if ab["attention"] > harness.L2_BYTES else \
+                  "inputs fit in L2 (%.1f MB per step): a correctness-sized workload, not flushed" % (ab["total"] / 1e6)
         line = {
             "metric": METRIC, "value": agg["us_per_step_job"], "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
             "ms_per_step": agg["ms_per_step"], "higher_is_better": False, "scaling": "weak", "vs_baseline": None,
@@ -389,15 +485,19 @@ def run_ours(args, w):
             "config": {"workload": w.name, "vocab": V, "k": w.k, "tree_nodes": N, "layers": L, "q_heads": Hq,
                        "kv_heads": Hkv, "head_dim": D, "context": list(w.ctx), "batch": B,
                        "attention_launch": "all layers in one launch",
-                       "l2": "inputs larger than L2: %.0f MB of K/V streamed per step" % (ab["attention"] / 1e6),
-                       "parallelism": "replicas only" if world > 1 else "1 gpu"},
+                       "graphs": "%d consecutive steps per CUDA graph launch, remaining steps one graph each" % n_rot,
+                       "l2": l2_note, "parallelism": "replicas only" if world > 1 else "1 gpu"},
+            "timing": {"blocks": len(block_ms), "steps_per_block": K, "value_is": "median block",
+                       "block_us_per_step_min": 1000.0 * min(block_ms) / K,
+                       "block_us_per_step_max": 1000.0 * max(block_ms) / K,
+                       "timed_device_ms": float(sum(block_ms))},
             "steps_per_s": agg["steps_per_s"],
-            "step_hbm": {"algorithmic_bytes": ab["total"], "achieved_gbs": step_gbs, "frac_of_measured": step_gbs / peak,
-                         "frac_of_8tbs": step_gbs / 8000.0},
-            "roofline": {"kernel": "tree attention (all layers)", "bound": "hbm", "achieved": attn_gbs, "peak": peak,
-                         "unit": "GB/s", "frac": attn_gbs / peak, "peak_source": peak_src,
+            "step_hbm": {"algorithmic_bytes": ab["total"], "achieved_gbs": step_gbs,
+                         "frac_of_measured": step_gbs / hbm_peak, "frac_of_8tbs": step_gbs / 8000.0},
+            "roofline": {"kernel": "tree attention (all layers)", "bound": bound, "achieved": top["achieved"],
+                         "peak": top["peak"], "unit": top["unit"], "frac": top["frac"], "peak_source": peak_src,
                          "algorithmic_bytes_per_launch": ab["attention"], "avg_launch_ms": attn_ms,
-                         "traffic": NCU_TRAFFIC_BYTES.get(w.name)},
+                         "traffic": NCU_TRAFFIC_BYTES.get(w.name), "hbm": hbm, "tensor": tensor},
             "attention_per_layer_launches_ms": per_layer_ms,
             "cpu_baseline": {"value": cpu_us, "unit": UNIT, "cores": cpu_threads, "kind": "oracle", "sample": cpu_desc},
             "e2e": {"value": e2e["us_per_step_job"], "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
@@ -405,7 +505,8 @@ def run_ours(args, w):
             "gpu_launches": dw.kernels_per_step() * K,
             "clocks": clocks,
             "mean_new_tokens_per_step": n_new_sum / (B * n_stat),
-            "next_rows": {"lm_head_topk": dict(lm, frac=lm["achieved"] / peak, peak=peak),
+            "parity_checked": bool(parity and parity.get("ok")), "parity": parity,
+            "next_rows": {"lm_head_topk": dict(lm, frac=lm["achieved"] / hbm_peak, peak=hbm_peak),
                           "verify_update_sampled": sampled_verify},
             "device_flags": flags,
         }
@@ -431,6 +532,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama2-7b")
     ap.add_argument("--layers", type=int, default=0, help="override the number of layers (profiling small cases)")
+    ap.add_argument("--min-timed-ms", type=float, default=50.0,
+                    help="the K-step block is repeated until the timed blocks add up to this much device time (>= 5 blocks)")
     ap.add_argument("--profile", action="store_true",
                     help="only warm up and replay the step graph K times (for ncu); prints no bench line")
     ap.add_argument("--lm-head-only", action="store_true",

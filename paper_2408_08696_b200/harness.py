@@ -75,31 +75,43 @@ class DeviceWorkload:
             tr.tr_tree_attention(self.ctx, self.attn, stream)
         tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, stream)
 
+    def _capture_steps(self, s, side, rots):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=s):
+            for r in rots:
+                if self.attn is not None:
+                    side.wait_stream(s)
+                    self.patch(r, side)
+                    tr.tr_tree_attention(self.ctx, self.attn, s)
+                    s.wait_stream(side)
+                else:
+                    self.patch(r, s)
+                tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, s)
+        return g
+
     def capture_graphs(self):
-        """One CUDA graph per rotating logits buffer; replay graphs[i % n_rot] for step i = 0, 1, 2, ... in order.
-        Graph r holds the step's own kernels in a chain - attention, top-k, accept/update/retrieve - and, on a side
-        branch that joins the chain in front of the top-k kernel, the toy model's patch of buffer r for the tree
-        the previous step left (harness work: it stands for the rest of the model's forward pass, which produces
-        the logits while the step's attention runs)."""
-        graphs = []
-        s = torch.cuda.Stream(self.dev)
-        side = torch.cuda.Stream(self.dev)
+        """One CUDA graph per rotating logits buffer: graph r is one whole step on buffer r.  A step's own kernels form
+        a chain - attention, top-k, accept/update/retrieve - and, on a side branch that joins the chain in front of
+        the top-k kernel, the toy model patches buffer r for the tree the previous step left (harness work: it
+        stands for the rest of the model's forward pass, which produces the logits while the step's attention
+        runs).  Every graph reads the current tree, so the graphs may be replayed in any order; the checker follows
+        the same order of buffers."""
+        s, side = torch.cuda.Stream(self.dev), torch.cuda.Stream(self.dev)
         torch.cuda.synchronize(self.dev)
         with torch.cuda.stream(s):
-            for r in range(self.n_rot):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=s):
-                    if self.attn is not None:
-                        side.wait_stream(s)
-                        self.patch(r, side)
-                        tr.tr_tree_attention(self.ctx, self.attn, s)
-                        s.wait_stream(side)
-                    else:
-                        self.patch(r, s)
-                    tr.tr_verify_update(self.ctx, self.d_logits[r], self.d_tree, self.out_struct, s)
-                graphs.append(g)
+            graphs = [self._capture_steps(s, side, [r]) for r in range(self.n_rot)]
         torch.cuda.synchronize(self.dev)
         return graphs
+
+    def capture_round(self):
+        """One CUDA graph holding n_rot consecutive steps (buffers 0 .. n_rot-1): the steps follow one another
+        inside the graph, which spares the launch gap between separate graph launches."""
+        s, side = torch.cuda.Stream(self.dev), torch.cuda.Stream(self.dev)
+        torch.cuda.synchronize(self.dev)
+        with torch.cuda.stream(s):
+            g = self._capture_steps(s, side, list(range(self.n_rot)))
+        torch.cuda.synchronize(self.dev)
+        return g
 
     def reset(self):
         """Back to the state right after construction (matrices, first tree, un-patched logits), so that a loop can

@@ -27,11 +27,21 @@ def max_over_ranks(value, device="cpu"):
     return float(t.item())
 
 
-def aggregate(elapsed_ms, steps_per_rank, device="cpu"):
+def max_over_ranks_vec(values, device="cpu"):
+    """Element-wise largest value over all ranks of a list of floats (one entry per timed block)."""
+    if not (dist.is_available() and dist.is_initialized()):
+        return [float(v) for v in values]
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def aggregate(elapsed_ms, steps_per_rank, device="cpu", reduce=True):
     """Whole-job figures for `world` replicas that each ran `steps_per_rank` steps in `elapsed_ms` (this rank's
-    device time): the job takes the slowest rank's time and completes world * steps_per_rank steps."""
+    device time, or with reduce=False a time that already is the maximum over ranks): the job takes the slowest
+    rank's time and completes world * steps_per_rank steps."""
     _, n = world()
-    t_ms = max_over_ranks(elapsed_ms, device)
+    t_ms = max_over_ranks(elapsed_ms, device) if reduce else float(elapsed_ms)
     total_steps = n * steps_per_rank
     return {
         "n_ranks": n,
