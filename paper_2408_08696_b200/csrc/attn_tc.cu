@@ -47,6 +47,7 @@ struct TcParams {
   // are packed into common 128-row tiles (row = node * G + head-in-group), MT tiles per head unit; when the group
   // size does not divide 128, every query head is its own head unit (G = 1) and kv_div maps it to its KV head.
   int HU, G, g_shift, MT, kv_div;
+  int live_warps;  // softmax warps that own at least one real row in every unit (4 unless tiles are unpacked and N <= 96)
   uint32_t div_MT[2], div_S[2], div_HU[2], div_L[2], div_kv[2];  // (multiplier, shift) for exact u32 division
   int64_t os_b, os_h, os_t, os_l;
   float scale_log2;
@@ -194,11 +195,11 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       mbar_init(bar(BAR_QFULL + i), 1);
       mbar_init(bar(BAR_QEMPTY + i), 1);
       mbar_init(bar(BAR_SFULL + i), 1);
-      mbar_init(bar(BAR_PFULL + i), 128);
+      mbar_init(bar(BAR_PFULL + i), 32u * static_cast<uint32_t>(p.live_warps));
       mbar_init(bar(BAR_PVDONE + i), 1);
       mbar_init(bar(BAR_OFREE + i), 128);
       mbar_init(bar(BAR_OREADY + i), 1);
-      mbar_init(bar(BAR_LFULL + i), 128);
+      mbar_init(bar(BAR_LFULL + i), 32u * static_cast<uint32_t>(p.live_warps));
     }
     *s_abort = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -342,7 +343,10 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t lane_base = static_cast<uint32_t>((warp & 3) * 32) << 16;
     uint32_t anc[4];
     uint32_t ui = 0, g = 0;
-    bool ok = true;
+    // A warp whose 32 rows lie past the tree's last node in every unit (80 nodes leave rows 96..127 of an unpacked tile
+    // empty) is not counted by the barriers of this role and goes straight to the teardown: its scores, exponentials
+    // and P rows would never be used.
+    bool ok = (warp & 3) < p.live_warps;
     for (int u = blockIdx.x; u < p.n_units && ok; u += gridDim.x) {
       const Unit x = decode_unit(p, u, s_ctx);
       const int nt = x.t1 - x.t0;
@@ -355,7 +359,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const uint32_t ob = ui & 1u;
       for (int j = 0; j < nt && ok; ++j, ++g) {
         const uint32_t sb = g & 1u;
-        ok = mbar_wait<false>(bar(BAR_SFULL + sb), (g >> 1) & 1u, s_abort);
+        ok = mbar_wait<0>(bar(BAR_SFULL + sb), (g >> 1) & 1u, s_abort);
         ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
         if (!ok) break;
         tc_fence_after();
@@ -419,7 +423,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (__any_sync(0xFFFFFFFFu, need)) {
           // O of this unit holds tiles < j; PV(j-1) must have landed before it is rescaled
           const uint32_t pb = (g - 1u) & 1u;
-          ok = mbar_wait<false>(bar(BAR_PVDONE + pb), ((g - 1u) >> 1) & 1u, s_abort);
+          ok = mbar_wait<0>(bar(BAR_PVDONE + pb), ((g - 1u) >> 1) & 1u, s_abort);
           ok = __all_sync(0xFFFFFFFFu, ok);
           if (!ok) break;
           tc_fence_after();
@@ -463,7 +467,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       if (nt <= 0) continue;  // empty split: the epilogue warps write its (empty) partial
       // ---- hand the unit to the epilogue warps: row sum and reference maximum go through shared memory.  The
       //      slot was last read by the epilogue of unit ui-2, which signalled OFREE when it was done with it.
-      ok = mbar_wait<false>(bar(BAR_OFREE + ob), ((ui >> 1) & 1u) ^ 1u, s_abort);
+      ok = mbar_wait<0>(bar(BAR_OFREE + ob), ((ui >> 1) & 1u) ^ 1u, s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       s_lm[ob * 256 + r] = l;
@@ -497,7 +501,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         continue;
       }
       const uint32_t ob = ui & 1u, par = (ui >> 1) & 1u;
-      ok = mbar_wait<false>(bar(BAR_LFULL + ob), par, s_abort) && mbar_wait<false>(bar(BAR_OREADY + ob), par, s_abort);
+      ok = mbar_wait<0>(bar(BAR_LFULL + ob), par, s_abort) && mbar_wait<0>(bar(BAR_OREADY + ob), par, s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);
       if (!ok) break;
       tc_fence_after();
@@ -669,6 +673,7 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   p.HU = packed ? a->n_kv_heads : a->n_q_heads;
   p.kv_div = packed ? 1 : group;
   p.MT = (ctx->n_nodes * p.G + 127) / 128;
+  p.live_warps = (p.MT == 1 && p.G == 1) ? (ctx->n_nodes + 31) / 32 : 4;
   const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * p.HU * p.MT;
   if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;
   p.out = static_cast<__nv_bfloat16*>(a->out);

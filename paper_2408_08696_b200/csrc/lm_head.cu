@@ -173,7 +173,7 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     bool ok = true;
     for (int c = 0; c < n_chunks && ok; ++c) {
       const uint32_t buf = c & 1u;
-      ok = mbar_wait<true>(bar(LM_BAR_ACC_FULL + buf), (c >> 1) & 1u, s_abort);
+      ok = mbar_wait<40>(bar(LM_BAR_ACC_FULL + buf), (c >> 1) & 1u, s_abort);
       ok = __all_sync(0xFFFFFFFFu, ok);  // the TMEM loads below are warp-collective
       if (!ok) break;
       tc_fence_after();

@@ -33,15 +33,16 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
   return ok;
 }
 // Bounded wait.  Returns false (and raises the CTA's abort flag) if the phase never completes.
-// kBackoff: sleep a little between polls (the single-thread producer / MMA roles share their scheduler with a
-// softmax warp and should not take its issue slots).
-template <bool kBackoff = false>
+// kSleepNs > 0: sleep that long between polls - for waits whose wake-up is not on the critical path.  A polling warp
+// is not free: its try_wait instructions go through the SM's shared-memory pipeline, which the TMA writes and the
+// tensor core's operand reads use as well.
+template <int kSleepNs = 0>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    if (kBackoff) __nanosleep(40);
+    if (kSleepNs > 0) __nanosleep(kSleepNs);
     if ((i & 63u) == 0u) {
       if (*abort_flag) return false;
       if (clock64() - t0 > WAIT_LIMIT_CYCLES) break;
