@@ -687,6 +687,9 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   const float scale = a->scale != 0.f ? a->scale : 1.0f / sqrtf(static_cast<float>(a->head_dim));
   p.scale_log2 = scale * 1.4426950408889634f;
   p.S = tr_attention_pick_splits(ctx, a, static_cast<int>(base), BK, true);
+  // grouped-query shapes with at least two row tiles per KV head and enough work without splitting the keys: two
+  // tiles per CTA on one K/V stream
+  if (p.S == 1 && tr_attention_pair_applies(ctx, a)) return tr_launch_attention_pair(ctx, a, s);
   p.n_units = static_cast<int>(base * p.S);
   magic_u32(static_cast<uint32_t>(p.MT), p.div_MT);
   magic_u32(static_cast<uint32_t>(p.S), p.div_S);

@@ -70,6 +70,7 @@ static tr_status free_all(tr_ctx* c) {
   }
   cudaFree(c->d_attn_part_o);
   cudaFree(c->d_attn_part_ml);
+  cudaFree(c->d_attn_queue);
   cudaFree(c->d_flags);
   delete c;
   return TR_OK;
@@ -151,6 +152,8 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
 
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_o, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 128));
   TR_INIT_TRY(cudaMalloc(&c->d_attn_part_ml, sizeof(float) * ATTN_MAX_PART_SLOTS * ATTN_PART_ROWS * 2));
+  TR_INIT_TRY(cudaMalloc(&c->d_attn_queue, sizeof(unsigned int) * 2));
+  TR_INIT_TRY(cudaMemset(c->d_attn_queue, 0, sizeof(unsigned int) * 2));
   // streams and events of tr_step_host's copy pipeline
   TR_INIT_TRY(cudaStreamCreateWithFlags(&c->io_in, cudaStreamNonBlocking));
   TR_INIT_TRY(cudaStreamCreateWithFlags(&c->io_out, cudaStreamNonBlocking));
@@ -168,6 +171,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   {
     tr_status st = tr_attention_mma_setup();
     if (st == TR_OK) st = tr_attention_tc_setup();
+    if (st == TR_OK) st = tr_attention_pair_setup();
     if (st == TR_OK) st = tr_lm_head_setup();
     if (st != TR_OK) {
       free_all(c);

@@ -51,6 +51,7 @@ struct tr_ctx {
   int lm_parts_cap = 0;
   float* d_attn_part_o = nullptr;   // [slots][128][128]
   float* d_attn_part_ml = nullptr;  // [slots][128][2]
+  unsigned int* d_attn_queue = nullptr;  // [2] unit counter of the two-tiles-per-CTA attention kernel (clears itself)
   uint32_t* d_flags = nullptr;
   // tr_step_host: host->device and device->host copy streams and the events that chain them to the caller's stream
   cudaStream_t io_in = nullptr, io_out = nullptr;
@@ -116,6 +117,9 @@ tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream
 tr_status tr_attention_mma_setup();
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_tc_setup();
+bool tr_attention_pair_applies(const tr_ctx* ctx, const tr_attn_args* a);
+tr_status tr_launch_attention_pair(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
+tr_status tr_attention_pair_setup();
 void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
 tr_status tr_lm_head_setup();
 tr_status tr_launch_lm_head(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,

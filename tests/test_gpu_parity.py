@@ -264,6 +264,22 @@ def test_attention_group_sizes(harness, hq, hkv):
     _attention_case(harness, w, 2, splits=2)
 
 
+@pytest.mark.parametrize("hq,hkv,ctxs,L", [
+    (8, 1, (150,), 1),          # 8 heads per KV head: five row tiles = two pairs and a lone left-over tile
+    (8, 2, (100, 257), 2),      # 4 per KV head: three tiles = one pair per KV head + one twin of the two left-overs
+    (12, 3, (333,), 2),         # odd number of KV heads: pairs, one twin and one lone tile
+    (4, 2, (64,), 3),           # 2 per KV head: two tiles, pairs only; the prefix ends on a tile boundary
+    (8, 2, (0, 1, 63), 1),      # empty and tiny prefixes: the tree block alone spans two key tiles
+    (32, 8, (1200, 40), 2),     # the llama3-8b head layout, two sequences of very different length
+])
+def test_attention_two_tiles_per_cta_kernel(harness, hq, hkv, ctxs, L):
+    """The grouped-query kernel that runs two row tiles per CTA on one K/V stream (pair, twin and lone units, 64-key
+    tiles, dynamic unit queue), forced by asking for no KV split; every output row against the oracle."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=hq, n_kv_heads=hkv, ctx=ctxs)
+    _attention_case(harness, w, L, splits=1)
+    _attention_case(harness, w, L, splits=1)      # a second launch finds the unit counter cleared
+
+
 @pytest.mark.parametrize("head_dim", [128, 64])
 def test_attention_other_memory_layouts_and_explicit_scale(harness, tr, head_dim):
     """The same tensors in other layouts - token-major caches [B, L, R, Hkv, D], head-major queries and outputs
