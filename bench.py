@@ -205,11 +205,11 @@ def measure_lm_head(torch, tr, dw, w, dev, reps=20):
     e1.record()
     torch.cuda.synchronize()
     us = e0.elapsed_time(e1) / reps * 1000.0
-    passes = (rows + 127) // 128                               # the kernel streams the weight once per 128 rows
+    groups = (rows + 127) // 128                               # row groups: the CTAs of a vocabulary slice share it via L2
     byts = w.vocab * H * 2 + rows * H * 2 + rows * w.k * 4      # algorithmic: the weight ONCE, hidden states, output
     return {"us": us, "bound": "hbm", "achieved": byts / us / 1e3, "unit": "GB/s", "algorithmic_bytes": byts,
-            "weight_passes": passes, "weight_bytes_streamed": passes * w.vocab * H * 2,
-            "rows": rows, "hidden": H, "vocab": w.vocab, "gpu_launches": passes + 1,
+            "row_groups": groups, "weight_bytes_through_sms": groups * w.vocab * H * 2,
+            "rows": rows, "hidden": H, "vocab": w.vocab, "gpu_launches": 2,
             "device_flags": tr.tr_device_flags(dw.ctx)}
 
 

@@ -200,8 +200,9 @@ tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits, const flo
  *             layout of a linear layer's weight), row stride weight_stride elements.  Both 16-byte aligned, strides
  *             multiples of 8 and >= hidden_dim, hidden_dim a multiple of 8 (else TR_ERR_INVALID_ARG).  No NaN.
  * DEVICE out: d_topk_idx [rows, k] int32; d_topk_val [rows, k] fp32 (the accumulated logits at those indices) or NULL.
- * Rows are processed in groups of 128, each group with its own pass over the weight.  Allocates nothing, reads
- * nothing back, does not synchronise; uses scratch of the context (not re-entrant per context).
+ * Rows are processed in groups of 128; the CTAs that work on the same vocabulary slice for different groups run side
+ * by side, so the weight is fetched from HBM once and shared through L2.  Allocates nothing, reads nothing back, does
+ * not synchronise; uses scratch of the context (not re-entrant per context).
  */
 tr_status tr_lm_head_topk(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,
                           int64_t weight_stride, int32_t hidden_dim, int32_t* d_topk_idx, float* d_topk_val,

@@ -586,15 +586,23 @@ extern "C" int tr_debug_stamps_pair(unsigned long long* host) {
 }
 #endif
 
+static bool g_pair_usable = false;
+
 tr_status tr_attention_pair_setup() {
   TR_CUDA_TRY(cudaFuncSetAttribute(tr_attn_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+  // The kernel raises its softmax warps' register budget at run time; the request blocks until the CTA's pool (the
+  // registers the kernel was compiled to launch with, times its threads) has that much to give.  Use the kernel only
+  // if the compiled register count makes the pool large enough - otherwise the other attention kernel serves.
+  cudaFuncAttributes fa;
+  TR_CUDA_TRY(cudaFuncGetAttributes(&fa, tr_attn_pair_kernel));
+  g_pair_usable = fa.numRegs * NTHREADS >= 8 * 32 * REGS_SOFTMAX + 4 * 32 * REGS_CONTROL;
   return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
 }
 
 // Whether the two-tiles-per-CTA kernel applies: head_dim 128, a group size > 1 that divides 128, at least two row tiles
 // per KV head.  (It has no split-KV path: the caller uses it only when the launch has enough units without splitting.)
 bool tr_attention_pair_applies(const tr_ctx* ctx, const tr_attn_args* a) {
-  if (a->head_dim != HD) return false;
+  if (!g_pair_usable || a->head_dim != HD) return false;
   const int group = a->n_q_heads / a->n_kv_heads;
   if (group <= 1 || (128 % group) != 0) return false;
   return (ctx->n_nodes * group + 127) / 128 >= 2;

@@ -41,9 +41,10 @@ constexpr int LM_MERGE_THREADS = 256;
 constexpr int LM_MERGE_CAND = 256;
 
 struct LmParams {
-  u64* part;        // [rows of this group][parts][k], parts = 2 * CTAs
+  u64* part;        // [rows][parts][k], parts = 2 * vocabulary slices
   uint32_t* flags;
-  int R;            // rows in this group (<= 128)
+  int R;            // rows in all (groups of 128: CTA = (vocabulary slice, row group), the groups of a slice adjacent)
+  int groups;       // row groups
   int V, H;         // vocabulary size, hidden size
   int cols_per_cta; // vocabulary slice of one CTA
   int NC;           // width of a chunk = the MMA's N (a multiple of 16, <= 256)
@@ -79,8 +80,11 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
   auto bar = [&](int i) { return bars + static_cast<uint32_t>(i) * 8u; };
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
-  // this CTA's slice and its chunks: chunk c starts at v_begin + c * NC
-  const int v_begin = blockIdx.x * p.cols_per_cta;
+  // this CTA's slice, row group and chunks: chunk c starts at v_begin + c * NC.  The CTAs of one slice (one per row
+  // group) have neighbouring indices, run at the same time and stream the same weight rows: the first to ask brings
+  // them in from HBM, the others find them in L2.
+  const int slice = blockIdx.x / p.groups, row0 = (blockIdx.x - slice * p.groups) * 128;
+  const int v_begin = slice * p.cols_per_cta;
   const int v_end = min(p.V, v_begin + p.cols_per_cta);
   int n_chunks = 0;
   for (int c = 0; c < p.n_main; ++c) n_chunks += (v_begin + c * p.NC < v_end) ? 1 : 0;
@@ -111,7 +115,7 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // =========================== TMA producer ===========================
     if (lane == 0) {
       const uint64_t pol = l2_policy_evict_first();  // the weight is read once; the hidden states stay in L2
-      const int k_shift = static_cast<int>((blockIdx.x * 11u) % static_cast<uint32_t>(ksteps));
+      const int k_shift = static_cast<int>((static_cast<uint32_t>(slice) * 11u) % static_cast<uint32_t>(ksteps));
       uint32_t it = 0;
       bool ok = true;
       for (int c = 0; c < n_chunks && ok; ++c) {
@@ -126,8 +130,9 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
           // that the CTAs, whose slices are a fixed large stride apart, do not march through DRAM in lockstep
           int kq = ks + k_shift;
           kq = kq >= ksteps ? kq - ksteps : kq;
-          tma_load_2d_hint(dst + LM_A_BYTES, &map_b, bar(LM_BAR_FULL + s), kq * LM_BK, v0, pol);
-          tma_load_2d(dst, &map_a, bar(LM_BAR_FULL + s), kq * LM_BK, 0);
+          if (p.groups == 1) tma_load_2d_hint(dst + LM_A_BYTES, &map_b, bar(LM_BAR_FULL + s), kq * LM_BK, v0, pol);
+          else tma_load_2d(dst + LM_A_BYTES, &map_b, bar(LM_BAR_FULL + s), kq * LM_BK, v0);  // shared through L2
+          tma_load_2d(dst, &map_a, bar(LM_BAR_FULL + s), kq * LM_BK, row0);
         }
       }
     }
@@ -218,8 +223,8 @@ tr_lm_head_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         mbar_arrive(bar(LM_BAR_ACC_EMPTY + buf));
       }
     }
-    if (ok && r < p.R) {
-      u64* dst = p.part + (static_cast<size_t>(r) * p.parts + 2 * blockIdx.x + half) * p.k;
+    if (ok && row0 + r < p.R) {
+      u64* dst = p.part + (static_cast<size_t>(row0 + r) * p.parts + 2 * slice + half) * p.k;
 #pragma unroll
       for (int i = 0; i < KMAX; ++i)
         if (i < p.k) dst[i] = idx[i] >= 0 ? lm_key(val[i], static_cast<uint32_t>(idx[i])) : 0ull;
@@ -342,13 +347,14 @@ tr_status tr_lm_head_setup() {
   return get_encode_fn() ? TR_OK : TR_ERR_CUDA;
 }
 
-// Vocabulary slice per CTA (V spread over at most sm_count CTAs, a multiple of 16), cut into equal chunks of at most
-// 256 columns, and as many ring stages as fit.
-static void lm_partition(const tr_ctx* ctx, LmParams* p, int* n_cta) {
-  int w = (ctx->vocab + ctx->sm_count - 1) / ctx->sm_count;
+// Vocabulary slice per CTA (V spread over at most sm_count / groups slices, a multiple of 16), cut into equal chunks of
+// at most 256 columns, and as many ring stages as fit.
+static void lm_partition(const tr_ctx* ctx, int groups, LmParams* p, int* n_slices) {
+  const int max_slices = ctx->sm_count / groups > 0 ? ctx->sm_count / groups : 1;
+  int w = (ctx->vocab + max_slices - 1) / max_slices;
   w = (w + 15) / 16 * 16;
   p->cols_per_cta = w;
-  *n_cta = (ctx->vocab + w - 1) / w;
+  *n_slices = (ctx->vocab + w - 1) / w;
   p->n_main = (w + LM_MAX_NC - 1) / LM_MAX_NC;
   p->NC = ((w + p->n_main - 1) / p->n_main + 15) / 16 * 16;
   const int stage = LM_A_BYTES + p->NC * LM_BK * 2;
@@ -360,32 +366,31 @@ tr_status tr_launch_lm_head(tr_ctx* ctx, const void* d_hidden, int64_t hidden_st
                             cudaStream_t s) {
   const int rows = ctx->batch * ctx->n_nodes;
   LmParams p;
-  int n_cta = 0;
-  lm_partition(ctx, &p, &n_cta);
+  // rows beyond 128 form further row groups; a vocabulary slice is then worked on by one CTA per group at the same
+  // time, so that the weight still comes from HBM once
+  p.groups = (rows + 127) / 128;
+  if (p.groups > ctx->sm_count) return TR_ERR_UNSUPPORTED;
+  int n_slices = 0;
+  lm_partition(ctx, p.groups, &p, &n_slices);
   p.flags = ctx->d_flags;
   p.V = ctx->vocab;
   p.H = hidden_dim;
   p.k = ctx->k;
-  p.parts = 2 * n_cta;
+  p.R = rows;
+  p.parts = 2 * n_slices;
+  p.part = ctx->d_lm_part;
   if (p.parts > ctx->lm_parts_cap) return TR_ERR_UNSUPPORTED;
   if (static_cast<size_t>(p.parts) * p.k * sizeof(u64) > 40 * 1024) return TR_ERR_UNSUPPORTED;  // merge kernel's staging
-  CUtensorMap mb;
+  CUtensorMap ma, mb;
   if (!lm_encode_map(&mb, d_weight, static_cast<uint64_t>(hidden_dim), static_cast<uint64_t>(ctx->vocab), weight_stride,
-                     static_cast<uint32_t>(p.NC)))
+                     static_cast<uint32_t>(p.NC)) ||
+      !lm_encode_map(&ma, d_hidden, static_cast<uint64_t>(hidden_dim), static_cast<uint64_t>(rows), hidden_stride, 128))
     return TR_ERR_UNSUPPORTED;
-  // rows beyond 128 are handled in groups of 128, each with its own pass over the weight
-  for (int g0 = 0; g0 < rows; g0 += 128) {
-    p.R = rows - g0 < 128 ? rows - g0 : 128;
-    p.part = ctx->d_lm_part + static_cast<size_t>(g0) * p.parts * p.k;
-    CUtensorMap ma;
-    const __nv_bfloat16* hp = static_cast<const __nv_bfloat16*>(d_hidden) + static_cast<int64_t>(g0) * hidden_stride;
-    if (!lm_encode_map(&ma, hp, static_cast<uint64_t>(hidden_dim), static_cast<uint64_t>(p.R), hidden_stride, 128))
-      return TR_ERR_UNSUPPORTED;
-    if (ctx->k <= 8)
-      TR_CUDA_TRY(tr_launch_pdl(tr_lm_head_kernel<8>, dim3(n_cta), dim3(LM_THREADS), LM_SMEM_BYTES, s, ma, mb, p));
-    else
-      TR_CUDA_TRY(tr_launch_pdl(tr_lm_head_kernel<16>, dim3(n_cta), dim3(LM_THREADS), LM_SMEM_BYTES, s, ma, mb, p));
-  }
+  const dim3 grid(static_cast<unsigned>(n_slices * p.groups));
+  if (ctx->k <= 8)
+    TR_CUDA_TRY(tr_launch_pdl(tr_lm_head_kernel<8>, grid, dim3(LM_THREADS), LM_SMEM_BYTES, s, ma, mb, p));
+  else
+    TR_CUDA_TRY(tr_launch_pdl(tr_lm_head_kernel<16>, grid, dim3(LM_THREADS), LM_SMEM_BYTES, s, ma, mb, p));
   TR_CUDA_TRY(tr_launch_pdl(tr_lm_head_merge_kernel, dim3(rows), dim3(LM_MERGE_THREADS),
                             sizeof(u64) * p.parts * p.k, s, static_cast<const u64*>(ctx->d_lm_part), p.parts, p.k,
                             d_topk_idx, d_topk_val));
