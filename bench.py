@@ -516,11 +516,14 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
-# DRAM bytes (read + write) of one attention launch from the committed ncu capture (see profiles/), per workload.
+# DRAM bytes (read + write) of one attention launch from the committed ncu captures (see profiles/), per workload.
 NCU_TRAFFIC_BYTES = {
-    # profiles/tr_attn_tc_kernel_llama2-7b_16layers.md: (300.03 MB read + 4.92 MB written) per 16-layer launch,
+    # profiles/tr_attn_tc_kernel_llama2-7b_16layers.md: (300.07 MB read + 4.93 MB written) per 16-layer launch,
     # scaled to the 32 layers of one benchmark launch (traffic is proportional to the layers processed)
-    "llama2-7b": 2 * (300_028_928 + 4_923_136),
+    "llama2-7b": 2 * (300_067_584 + 4_926_464),
+    # profiles/tr_attn_pair_kernel_llama3-8b_12layers.md: (414.64 MB read + 3.81 MB written) per 12-layer launch,
+    # scaled to 32 layers
+    "llama3-8b": int(round(32 / 12 * (414_638_080 + 3_806_208))),
 }
 
 
