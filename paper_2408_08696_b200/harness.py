@@ -22,7 +22,8 @@ def rotation_larger_than_l2(w: synth.Workload, factor=1.5):
     """Number of rotating logits buffers whose total size exceeds `factor` x the L2 capacity, so that in a loop that
     cycles through them every step's logits come from HBM, not from a warm L2 (at least 4)."""
     per_step = w.batch * w.n_nodes * w.vocab * 4
-    return max(4, -(-int(factor * L2_BYTES) // per_step))
+    n = max(4, -(-int(factor * L2_BYTES) // per_step))
+    return n if n <= 64 else 4      # a workload this small lives in L2 whatever is rotated
 
 
 class DeviceWorkload:
