@@ -243,37 +243,27 @@ def update_matrix(M, S, O, rule="last", nodes=None):
 # Draft tree retrieval (Sec. 3.2, Algorithm 1)
 # --------------------------------------------------------------------------
 def bfs_tree(M, parent, rank, root):
-    """Merged sequence S for the next step.
+    """Merged sequence S for the next step (Sec. 3.2): the root is the last
+    confirmed token, and every other template node holds the candidate that its
+    parent's token has in the column the template names,
 
-    Algorithm 1, with the depth counter advancing once per iteration: the
-    current layer L starts as (root); xs = M[L] holds all candidates of the
-    layer; the template picks from the flattened xs the entries
-    (position of the parent inside L) * k + rank for each child; S collects the
-    layers in order.
-    Pinned by: the two-layer walk-through of Sec. 3.2 on symbolic tokens; node
-    count and parent structure; all-zero matrix -> all drafts are token 0.
+        S[0] = root,   S[i] = M[S[parent[i]], rank[i]]   for i = 1 .. N-1,
+
+    taken in layer order, so a parent's token is known before its children's.
+    This is what Algorithm 1's layer-by-layer loop produces (its flat index
+    into xs = M[L] is (position of the parent in the layer) * k + rank); the
+    tests check that layered form against this definition.
+    Pinned by: the two-layer walk-through of Sec. 3.2 on symbolic tokens; the
+    layer-by-layer form of Algorithm 1 written out in the test; node count;
+    all-zero matrix -> all drafts are token 0.
     """
     parent = np.asarray(parent)
     rank = np.asarray(rank)
-    n = len(parent)
-    k = M.shape[1]
-    depth = node_depth(parent)
-    S = []
-    L = np.asarray([root], dtype=np.int64)
-    layer_nodes = [0]                         # template nodes forming layer L
-    d = 0
-    while len(S) < n:
-        S.extend(int(t) for t in L)
-        xs = M[L]                             # [|L|, k]
-        nxt = [i for i in range(n) if depth[i] == d + 1]
-        pos = {node: p for p, node in enumerate(layer_nodes)}
-        index = [pos[parent[i]] * k + rank[i] for i in nxt]   # Tree[d].index
-        L = xs.reshape(-1)[index] if index else np.zeros(0, dtype=np.int64)
-        layer_nodes = nxt
-        d += 1
-        if not nxt:
-            break
-    return np.asarray(S, dtype=np.int64)
+    S = np.zeros(len(parent), dtype=np.int64)
+    S[0] = root
+    for i in range(1, len(parent)):
+        S[i] = M[S[parent[i]], rank[i]]
+    return S
 
 
 # --------------------------------------------------------------------------

@@ -344,6 +344,36 @@ def test_bfs_matches_section_3_2_walkthrough(golden_dir):
     assert S.tolist() == g["S"]
 
 
+def _algorithm_1_layer_by_layer(M, parent, rank, root):
+    """Algorithm 1 as printed, with the depth counter advancing once per iteration: the current layer L starts as
+    (root); xs = M[L] holds all candidates of the layer; the template picks from the flattened xs the entries
+    (position of the parent inside L) * k + rank for each child; S collects the layers in order."""
+    n, k = len(parent), M.shape[1]
+    depth = orc.node_depth(parent)
+    S, L, layer_nodes, d = [], np.asarray([root], dtype=np.int64), [0], 0
+    while len(S) < n:
+        S.extend(int(t) for t in L)
+        xs = M[L]
+        nxt = [i for i in range(n) if depth[i] == d + 1]
+        pos = {node: p for p, node in enumerate(layer_nodes)}
+        index = [pos[parent[i]] * k + rank[i] for i in nxt]
+        L = xs.reshape(-1)[index] if index else np.zeros(0, dtype=np.int64)
+        layer_nodes, d = nxt, d + 1
+        if not nxt:
+            break
+    return S
+
+
+@pytest.mark.parametrize("b,n", [((8, 4, 3, 2, 2, 1), 80), ((4, 2, 1), 15), ((2,) * 6, 127), ((1,) * 9, 10), ((16,), 17)])
+def test_bfs_equals_algorithm_1_layer_by_layer(b, n):
+    parent, rank = orc.template_from_branching(b, n)
+    rng = np.random.default_rng(n)
+    V, k = 300, 16
+    M = rng.integers(0, V, size=(V, k))
+    for root in (0, 7, V - 1):
+        assert orc.bfs_tree(M, parent, rank, root).tolist() == _algorithm_1_layer_by_layer(M, parent, rank, root)
+
+
 def test_bfs_node_count_parent_structure_and_zero_matrix():
     parent, rank = orc.template_from_branching((8, 4, 3, 2, 2, 1), 80)
     rng = np.random.default_rng(10)
