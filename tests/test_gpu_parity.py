@@ -264,6 +264,17 @@ def test_attention_group_sizes(harness, hq, hkv):
     _attention_case(harness, w, 2, splits=2)
 
 
+def test_attention_two_tiles_per_cta_kernel_largest_tree_and_wide_groups(harness):
+    """128 nodes with 4 heads per KV head (four full row tiles = two pair units per KV head), and 16 / 32 heads per KV
+    head (8 / 4 nodes per tile; ten and twenty row tiles) on the default tree."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], branching=(10, 10), n_nodes=128, n_q_heads=8, n_kv_heads=2,
+                            ctx=(200, 77), vocab=3000, k=16)
+    _attention_case(harness, w, 2, splits=1)
+    for hq, hkv in ((16, 1), (32, 1)):
+        w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=hq, n_kv_heads=hkv, ctx=(150,))
+        _attention_case(harness, w, 1, splits=1)
+
+
 @pytest.mark.parametrize("hq,hkv,ctxs,L", [
     (8, 1, (150,), 1),          # 8 heads per KV head: five row tiles = two pairs and a lone left-over tile
     (8, 2, (100, 257), 2),      # 4 per KV head: three tiles = one pair per KV head + one twin of the two left-overs
@@ -303,7 +314,7 @@ def test_attention_other_memory_layouts_and_explicit_scale(harness, tr, head_dim
     o_hm = torch.zeros_like(q_hm)
     q_view, o_view = q_hm.permute(0, 1, 3, 2, 4), o_hm.permute(0, 1, 3, 2, 4)
     d_ctx = torch.tensor(list(w.ctx), dtype=torch.int32, device="cuda")
-    for splits in (0, 2):
+    for splits in (0, 2, 1):        # 1: no KV split - at head_dim 128 the two-tiles-per-CTA kernel (2 heads per KV head)
         o_hm.zero_()
         a = tr.make_attn_args(ctx, q_view, k_view, v_view, o_view, d_ctx, w.max_ctx, scale=scale, splits=splits)
         tr.tr_tree_attention(ctx, a)
