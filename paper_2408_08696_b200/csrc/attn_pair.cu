@@ -307,6 +307,9 @@ tr_attn_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         ok = mbar_wait<0>(bar(BAR_QFULL + s), us & 1u, s_abort);
         if (!ok) break;
         ok = issue_qk(c + 2u * src, x.shared != 0);
+        // (the Q tile is handed back as soon as the unit's last S = Q K^T has been issued, so that the next unit's Q
+        // arrives under this unit's last tile)
+        if (x.nt == 1) tc_commit(bar(BAR_QEMPTY + s));
         for (int t = 0; t < x.nt && ok; ++t, ++g) {
           if (t == 0) {  // the accumulator must have been read out by the stream's epilogue of its previous unit
             ok = mbar_wait<0>(bar(BAR_OFREE + s), (us & 1u) ^ 1u, s_abort);
@@ -339,13 +342,13 @@ tr_attn_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
           c += 2u * nsrc;
           ++n_t;
           if (t == x.nt - 1) {
-            tc_commit(bar(BAR_QEMPTY + s));  // every QK of the unit has been issued: the Q tile is free when they finish
             tc_commit(bar(BAR_OREADY + s));  // the stream's output is complete
             ++us;
             PACC(w_pvi, t0);
           } else {
             PACC(w_pvi, t0);
             ok = issue_qk(c + 2u * src, x.shared != 0);  // the next tile's scores, right behind this tile's PV
+            if (t == x.nt - 2) tc_commit(bar(BAR_QEMPTY + s));  // that was the unit's last S = Q K^T
           }
         }
       }
