@@ -14,7 +14,7 @@ INCLUDE = os.path.join(ROOT, "include")
 LIB_TR = os.path.join(PKG, "libtr.so")
 LIB_SYNTH = os.path.join(PKG, "libtr_synth.so")
 
-TR_SOURCES = ["tr_api.cu", "topk.cu", "topk_noalloc.cu", "tail.cu", "attn_mma.cu", "attn_tc.cu", "attn_pair.cu", "commit.cu", "lm_head.cu"]
+TR_SOURCES = ["tr_api.cu", "topk.cu", "topk_noalloc.cu", "tail.cu", "attn_tc.cu", "attn_pair.cu", "commit.cu", "lm_head.cu"]
 SYNTH_SOURCES = ["synth.cu"]
 
 NVCC_FLAGS = [

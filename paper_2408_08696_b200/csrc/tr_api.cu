@@ -169,8 +169,7 @@ extern "C" tr_status tr_init(tr_ctx** out, int32_t vocab, int32_t k, const int32
   TR_INIT_TRY(cudaDeviceSynchronize());
 #undef TR_INIT_TRY
   {
-    tr_status st = tr_attention_mma_setup();
-    if (st == TR_OK) st = tr_attention_tc_setup();
+    tr_status st = tr_attention_tc_setup();
     if (st == TR_OK) st = tr_attention_pair_setup();
     if (st == TR_OK) st = tr_lm_head_setup();
     if (st != TR_OK) {
@@ -341,9 +340,7 @@ static tr_status check_attn_args(const tr_ctx* ctx, const tr_attn_args* a) {
 extern "C" tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* a, void* stream) {
   tr_status st = check_attn_args(ctx, a);
   if (st != TR_OK) return st;
-  // head_dim 128 runs on the tcgen05 / TMA kernel; head_dim 64 on the warp-level MMA kernel
-  if (a->head_dim == 128) return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
-  return tr_launch_attention_mma(ctx, a, static_cast<cudaStream_t>(stream));
+  return tr_launch_attention_tc(ctx, a, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" tr_status tr_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,

@@ -113,15 +113,12 @@ tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* 
 tr_status tr_launch_commit(tr_ctx* ctx, const tr_commit_args* a, const int32_t* d_acc_nodes,
                            const int32_t* d_out_tokens, const int32_t* d_n_new, cudaStream_t s);
 tr_status tr_launch_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, cudaStream_t s);
-tr_status tr_launch_attention_mma(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
-tr_status tr_attention_mma_setup();
 tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_tc_setup();
 bool tr_attention_pair_applies(const tr_ctx* ctx, const tr_attn_args* a);
 tr_status tr_launch_attention_pair(tr_ctx* ctx, const tr_attn_args* a, cudaStream_t s);
 tr_status tr_attention_pair_setup();
-void tr_launch_attention_combine(tr_ctx* ctx, const tr_attn_args* a, int S, cudaStream_t s);
 tr_status tr_lm_head_setup();
 tr_status tr_launch_lm_head(tr_ctx* ctx, const void* d_hidden, int64_t hidden_stride, const void* d_weight,
                             int64_t weight_stride, int hidden_dim, int32_t* d_topk_idx, float* d_topk_val, cudaStream_t s);
-int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys, bool fill_once);
+int tr_attention_pick_splits(const tr_ctx* ctx, const tr_attn_args* a, int base_units, int tile_keys);
