@@ -115,6 +115,8 @@ tr_status tr_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, voi
  * All base pointers 16-byte aligned and all strides multiples of 8 elements.
  * n_layers > 1 runs that many independent layers in one launch (layers of a real model are sequential;
  * this is for callers that hold all layers' q already, e.g. benchmarks).
+ * The call uses scratch of the context (split-KV partials, a unit counter): calls on one context must not overlap
+ * on the device (one stream, or streams ordered by events).
  * Errors: TR_ERR_INVALID_ARG (NULL, bad head counts, alignment), TR_ERR_UNSUPPORTED (head_dim not 64/128).
  */
 typedef struct {

@@ -93,7 +93,11 @@ __device__ __forceinline__ unsigned long long tr_globaltimer() {
 }
 // "MIN": the first CTA's time of the latest launch (plain store); "MAX": the latest time over all CTAs so far
 #define TR_STAMP_MIN(arr, i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) arr[i] = tr_globaltimer(); } while (0)
+#ifdef TR_STAMPS_NOMAX  // only the first CTA's plain stores: no atomics that could disturb what is being timed
+#define TR_STAMP_MAX(arr, i) do { } while (0)
+#else
 #define TR_STAMP_MAX(arr, i) do { if (threadIdx.x == 0) atomicMax(&arr[i], tr_globaltimer()); } while (0)
+#endif
 #endif
 #else
 #define TR_STAMP_DECL(name, n)
