@@ -56,6 +56,7 @@ def test_host_side_argument_errors(tr):
     assert init(100, 0, p, r, 15) == tr.TR_ERR_INVALID_ARG
     assert init(100, 17, p, r, 15) == tr.TR_ERR_INVALID_ARG
     assert init(100, 8, p, r, 15, batch=0) == tr.TR_ERR_INVALID_ARG
+    assert init(100, 8, p, r, 15, batch=4370) == tr.TR_ERR_UNSUPPORTED    # batch * nodes = 65550 logits rows: a grid's y limit
     assert init(100, 8, p, r, 0) == tr.TR_ERR_TEMPLATE
     assert init(100, 8, p, r, 129) == tr.TR_ERR_TEMPLATE
     bad = p.copy(); bad[3] = 7
@@ -70,6 +71,8 @@ def test_host_side_argument_errors(tr):
     assert tr.lib.tr_tree_attention(None, None, None) == tr.TR_ERR_INVALID_ARG
     assert tr.lib.tr_verify_update(None, None, None, None, None) == tr.TR_ERR_INVALID_ARG
     assert tr.lib.tr_destroy(None) == tr.TR_ERR_INVALID_ARG
+    assert tr.lib.tr_matrix_fill(None, 0, 0, None) == tr.TR_ERR_INVALID_ARG
+    assert tr.lib.tr_set_update_rule(None, 0, 0) == tr.TR_ERR_INVALID_ARG
     assert tr.lib.tr_status_string(tr.TR_ERR_TEMPLATE) == b"malformed tree template"
     with pytest.raises(tr.TrError):
         tr.tr_template_from_branching((4, 2, 1), 1000)
