@@ -15,8 +15,8 @@
 //   part list : candidates ranked by counting (four threads per candidate) -> the part's k best keys, stored straight
 //               into the shared memory of EVERY CTA of the cluster (distributed shared memory)
 //   merge     : after one cluster barrier every CTA holds all P lists and ranks its own k keys among them by counting
-//               (eight threads per key); a key with fewer than k keys above it is written to its place of the row's
-//               top-k.  Keys are distinct, so the P CTAs write disjoint places.
+//               (four threads per key; the other warps have left by then); a key with fewer than k keys above it is
+//               written to its place of the row's top-k.  Keys are distinct, so the P CTAs write disjoint places.
 // No global scratch, no atomics on global memory, no second kernel.  Massive ties (more candidates than the buffer
 // holds) take an exact, slower path that selects round by round from global memory.
 #include "tr_internal.cuh"
@@ -262,29 +262,37 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
   if (P > 1) {
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     TR_STAMP_MIN(g_stamps, 10);
+    // The final ranking takes 4 threads per key.  Threads without a key leave here: a warp that waits at the cluster
+    // barrier is not idle for the SM's schedulers, and with four or five CTAs per SM the waiting warps slowed the
+    // working ones down (1.6 us of the kernel at 80 rows x 32000).
+    if (tid >= 4 * (k <= 8 ? 8 : TR_MAX_K)) return;
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   } else {
     __syncthreads();
   }
   TR_STAMP_MIN(g_stamps, 11);
   TR_STAMP_MAX(g_stamps, 4);
-  {
-    // eight threads per key: thread (i, q) counts the keys of list q above key i of this part's list
-    const int i = tid >> 3, q = tid & 7;
+  if (tid < 4 * (k <= 8 ? 8 : TR_MAX_K)) {
+    // four threads per key: thread (i, q) counts the keys of lists q and q + 4 above key i of this part's list (every
+    // list has TR_MAX_K entries, zeros behind its k keys; with k <= 8 the first half of a list is enough)
+    const int i = tid >> 2, q = tid & 3;
     const u64 mine = my_list[i];
     int larger = 0;
-    if (q < P) {
-      const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(s_all + q * TR_MAX_K);
-      const ulonglong2 a0 = lp[0], a1 = lp[1], a2 = lp[2], a3 = lp[3];
-      larger = count_gt(a0, mine) + count_gt(a1, mine) + count_gt(a2, mine) + count_gt(a3, mine);
-      if (k > 8) {
-        const ulonglong2 a4 = lp[4], a5 = lp[5], a6 = lp[6], a7 = lp[7];
-        larger += count_gt(a4, mine) + count_gt(a5, mine) + count_gt(a6, mine) + count_gt(a7, mine);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int ql = q + 4 * h;
+      if (ql < P) {
+        const ulonglong2* lp = reinterpret_cast<const ulonglong2*>(s_all + ql * TR_MAX_K);
+        const ulonglong2 a0 = lp[0], a1 = lp[1], a2 = lp[2], a3 = lp[3];
+        larger += count_gt(a0, mine) + count_gt(a1, mine) + count_gt(a2, mine) + count_gt(a3, mine);
+        if (k > 8) {
+          const ulonglong2 a4 = lp[4], a5 = lp[5], a6 = lp[6], a7 = lp[7];
+          larger += count_gt(a4, mine) + count_gt(a5, mine) + count_gt(a6, mine) + count_gt(a7, mine);
+        }
       }
     }
     larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 1);
     larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 2);
-    larger += __shfl_xor_sync(0xFFFFFFFFu, larger, 4);
     if (q == 0 && mine != 0ull && larger < k)
       topk_idx[static_cast<size_t>(row) * k + larger] = static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(mine));
   }

@@ -87,9 +87,13 @@ __device__ __forceinline__ void tr_grid_dependency_wait() { asm volatile("gridde
 #define TR_STAMP_DECL(name, n) static __device__ unsigned long long name[n];
 #ifdef __CUDACC__
 __device__ __forceinline__ unsigned long long tr_globaltimer() {
+#ifdef TR_STAMPS_CLK  // SM cycle counter instead of the global timer: only differences inside one CTA mean anything
+  return static_cast<unsigned long long>(clock64());
+#else
   unsigned long long t;
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
+#endif
 }
 // "MIN": the first CTA's time of the latest launch (plain store); "MAX": the latest time over all CTAs so far
 #define TR_STAMP_MIN(arr, i) do { if (threadIdx.x == 0 && blockIdx.x == 0 && blockIdx.y == 0) arr[i] = tr_globaltimer(); } while (0)
