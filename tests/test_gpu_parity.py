@@ -209,6 +209,77 @@ def test_duplicate_tokens_last_writer_wins(tr):
     tr.tr_destroy(ctx)
 
 
+def _random_template(rng, n, k):
+    """An irregular static tree in level order: every node draws its own number of children (ranks 0..c-1)."""
+    parent, rank, level = [-1], [0], [0]
+    while len(parent) < n:
+        nxt = []
+        for p_ in level:
+            for r in range(int(rng.integers(0, min(k, 4) + 1))):
+                if len(parent) < n:
+                    parent.append(p_)
+                    rank.append(r)
+                    nxt.append(len(parent) - 1)
+        if not nxt:                                    # nobody drew a child: the level's first node gets one
+            parent.append(level[0])
+            rank.append(0)
+            nxt.append(len(parent) - 1)
+        level = nxt
+    return np.array(parent, dtype=np.int32), np.array(rank, dtype=np.int32)
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_verify_update_seeded_random_configurations(tr, seed):
+    """Irregular templates (children counts differ inside a level), small vocabularies (duplicate tokens in the tree),
+    tie-heavy integer logits with planted continuations, every update rule and scope, 1-4 sequences: three chained
+    steps each, every integer output and the matrix against the oracle."""
+    rng = np.random.default_rng(7000 + seed)
+    k = int(rng.choice([1, 2, 4, 5, 8, 12, 16]))
+    n = int(rng.choice([1, 2, 7, 31, 80, 97, 128]))
+    V = int(rng.choice([max(k, 16), 97, 1000, 4099]))
+    B = int(rng.integers(1, 5))
+    rule = ["last", "first"][int(rng.integers(2))]
+    only_accepted = bool(rng.integers(2))
+    parent, rank = _random_template(rng, n, k)
+    ctx = tr.tr_init(V, k, parent, rank, batch=B)
+    tr.tr_set_update_rule(ctx, tr.TR_UPDATE_FIRST if rule == "first" else tr.TR_UPDATE_LAST,
+                          tr.TR_UPDATE_ONLY_ACCEPTED if only_accepted else tr.TR_UPDATE_ALL_DRAFT)
+    M = [rng.integers(0, V, size=(V, k)).astype(np.int32) for _ in range(B)]
+    for b in range(B):
+        tr.tr_matrix_import(ctx, b, M[b])
+    roots = rng.integers(0, V, size=B).astype(np.int32)
+    d_tree = torch.zeros(B, n, dtype=torch.int32, device="cuda")
+    tr.tr_build_tree(ctx, torch.from_numpy(roots).cuda(), d_tree)
+    S = d_tree.cpu().numpy().copy()
+    for b in range(B):
+        assert (S[b] == orc.bfs_tree(M[b], parent, rank, int(roots[b]))).all()
+    out_struct, out = tr.make_step_out(ctx)
+    children = [[j for j in range(n) if parent[j] == i] for i in range(n)]
+    for step in range(3):
+        logits = rng.integers(-3, 4, size=(B, n, V)).astype(np.float32)
+        for b in range(B):
+            for i in range(n):
+                if children[i] and rng.random() < 0.6:        # the model "agrees" with one of the node's drafts
+                    logits[b, i, S[b, children[i][int(rng.integers(len(children[i])))]]] += 10.0
+        tr.tr_verify_update(ctx, torch.from_numpy(logits).cuda(), d_tree, out_struct)
+        torch.cuda.synchronize()
+        got = {name: t.cpu().numpy() for name, t in out.items()}
+        for b in range(B):
+            rec = orc.verify_update(M[b], S[b], logits[b], parent, rank, rule=rule, only_accepted=only_accepted)
+            m = rec["n_new"]
+            assert (got["topk_idx"][b] == rec["topk"]).all()
+            assert got["n_new"][b] == m
+            assert got["acc_nodes"][b, :m].tolist() == rec["acc_nodes"]
+            assert got["out_tokens"][b, :m].tolist() == rec["out_tokens"]
+            assert got["next_root"][b] == rec["next_root"]
+            assert (got["next_tree"][b] == rec["next_tree"]).all()
+            assert (tr.tr_matrix_export(ctx, b) == M[b]).all()
+            S[b] = rec["next_tree"]
+        d_tree.copy_(out["next_tree"])
+    assert tr.tr_device_flags(ctx) == 0
+    tr.tr_destroy(ctx)
+
+
 # ------------------------------------------------------------------ tree attention
 def _attention_case(harness, w, n_layers, splits=0):
     dw = harness.DeviceWorkload(w, n_layers=n_layers, splits=splits)
