@@ -34,16 +34,15 @@ __device__ __forceinline__ void load_tables(TailTables& t, int n, int depth_max,
   for (int i = tid; i < depth_max + 2; i += TAIL_THREADS) t.level_off[i] = level_off[i];
 }
 
-__device__ __forceinline__ void bfs_expand(const int32_t* __restrict__ M, int V, int k, int n,
-                                           const int32_t* parent, const int32_t* rank,
-                                           const int32_t* level_off, int depth_max,
+// One dependent round of gathers per level; every node of a level is looked up in parallel.  Thread i is node i and
+// holds its parent, rank and depth in registers (depth -1: no node), so that a level's chain is just barrier -> parent's
+// token from shared memory -> the gather -> store.
+__device__ __forceinline__ void bfs_expand(const int32_t* __restrict__ M, int k, int my_parent, int my_rank,
+                                           int my_depth, int depth_max,
                                            int32_t* s_tree /* shared [n], s_tree[0] set */, int tid) {
-  // one dependent round of gathers per level; every node of a level is looked up in parallel
   for (int d = 1; d <= depth_max; ++d) {
     __syncthreads();
-    const int lo = level_off[d], hi = level_off[d + 1];
-    const int i = lo + tid;
-    if (i < hi) s_tree[i] = __ldcg(M + static_cast<size_t>(s_tree[parent[i]]) * k + rank[i]);
+    if (d == my_depth) s_tree[tid] = __ldcg(M + static_cast<size_t>(s_tree[my_parent]) * k + my_rank);
   }
   __syncthreads();
 }
@@ -65,7 +64,12 @@ tr_build_tree_kernel(const int32_t* __restrict__ M_all, int V, int k, int n, con
     }
     s_tree[0] = r;
   }
-  bfs_expand(M, V, k, n, tb.parent, tb.rank, tb.level_off, depth_max, s_tree, tid);
+  __syncthreads();
+  int my_depth = -1;  // (this kernel gets no depth table: the level whose range holds the node)
+  if (tid < n)
+    for (int d = 0; d <= depth_max; ++d)
+      if (tid >= tb.level_off[d] && tid < tb.level_off[d + 1]) my_depth = d;
+  bfs_expand(M, k, tid < n ? tb.parent[tid] : 0, tid < n ? tb.rank[tid] : 0, my_depth, depth_max, s_tree, tid);
   if (tid < n) tree[static_cast<size_t>(b) * n + tid] = s_tree[tid];
 }
 
@@ -90,6 +94,9 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // ---- static tables (written by tr_init): fetched while the kernel in front may still be running
   load_tables(tb, n, depth_max, parent, rank, depth, level_off, tid);
+  // (this thread's own entries, for the retrieval at the end)
+  const int my_parent = tid < n ? tb.parent[tid] : 0, my_rank = tid < n ? tb.rank[tid] : 0;
+  const int my_depth = tid < n ? tb.depth[tid] : -1;
   uint32_t my_anc[4] = {0u, 0u, 0u, 0u};  // bit j: node j is this node or one of its ancestors
   if (tid < n) {
     const uint4 a = *reinterpret_cast<const uint4*>(anc + tid * 4);
@@ -219,7 +226,7 @@ tr_tail_kernel(int32_t* __restrict__ M_all, int V, int k, int n, const int32_t* 
   }
   TR_STAMP_MAX(g_tail_stamps, 4);
   // ---- retrieve the next tree from the updated matrix (bfs_expand starts with a __syncthreads())
-  bfs_expand(M, V, k, n, tb.parent, tb.rank, tb.level_off, depth_max, s_tree, tid);
+  bfs_expand(M, k, my_parent, my_rank, my_depth, depth_max, s_tree, tid);
   if (tid < n) tree_out[static_cast<size_t>(b) * n + tid] = s_tree[tid];
   TR_STAMP_MAX(g_tail_stamps, 5);
 }
