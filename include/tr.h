@@ -184,7 +184,8 @@ tr_status tr_verify_update_topk(tr_ctx* ctx, const int32_t* d_tree, const tr_ste
  * DEVICE in : d_logits, d_gumbel [batch, N, V] fp32 (the noise is the caller's: any generator, one row per node);
  *             inv_temperature > 0 and finite (else TR_ERR_INVALID_ARG); d_tree [batch, N].
  * DEVICE out: as tr_verify_update; d_sampled [batch, N] int32 receives the draws (NULL: kept in the context).
- * Two passes over the logits and one over the noise; allocates nothing, does not synchronise.
+ * Two passes over the logits and one over the noise, side by side in one launch (two clusters per row: top-k and
+ * draw); 2 * batch * n_nodes must not exceed 65535 (TR_ERR_UNSUPPORTED).  Allocates nothing, does not synchronise.
  */
 tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits, const float* d_gumbel, float inv_temperature,
                                    const int32_t* d_tree, const tr_step_out* out, int32_t* d_sampled, void* stream);

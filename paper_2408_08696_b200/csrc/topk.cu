@@ -65,13 +65,16 @@ __device__ __forceinline__ void st_all_u64(const void* p, u64 v, int n_ctas) {
 }
 __device__ __forceinline__ int count_gt(const ulonglong2& a, u64 x) { return (a.x > x) + (a.y > x); }
 
-// kSample: rank z = fl32(fl32(logit * inv_t) + gumbel) instead of the logits (Sec. 5.3 temperature sampling: with k = 1
-// the result is the token drawn at temperature 1 / inv_t by the Gumbel-max rule).  Two roundings, no fused multiply-add:
-// the decision is reproducible with plain float32 arithmetic.
+// kSample: the clusters blockIdx.y >= rows_plain rank z = fl32(fl32(logit * inv_t) + gumbel) instead of the logits
+// (Sec. 5.3 temperature sampling: with k = 1 the result is the token drawn at temperature 1 / inv_t by the Gumbel-max
+// rule) and write their k_sample best to out_sample.  Two roundings, no fused multiply-add: the decision is
+// reproducible with plain float32 arithmetic.  rows_plain = 0: every cluster samples; rows_plain = rows with 2 * rows
+// clusters: the model's top-k and the draw of every row in one launch, side by side.
 template <bool kVec, bool kSample>
 __global__ void __launch_bounds__(KT)
-tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_part, int32_t* __restrict__ topk_idx,
-               const float* __restrict__ gumbel, float inv_t) {
+tr_topk_kernel(const float* __restrict__ logits, int V, int k_plain, int chunks_per_part,
+               int32_t* __restrict__ out_plain, const float* __restrict__ gumbel, float inv_t, int rows_plain,
+               int k_sample, int32_t* __restrict__ out_sample) {
   __shared__ __align__(16) u64 s_cand[CAND_CAP + 32];        // candidates, then up to 32 zeros of padding
   __shared__ __align__(16) u64 s_all[MAX_PARTS * TR_MAX_K];  // every part's list (each CTA gets a copy)
   __shared__ u64 s_red[KT / 32];
@@ -79,7 +82,11 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
   __shared__ uint32_t s_tau;
   __shared__ int s_cnt;
 
-  const int part = blockIdx.x, P = gridDim.x, row = blockIdx.y;
+  const int part = blockIdx.x, P = gridDim.x;
+  const bool sample = kSample && static_cast<int>(blockIdx.y) >= rows_plain;  // the same for a whole cluster
+  const int row = sample ? blockIdx.y - rows_plain : blockIdx.y;
+  const int k = sample ? k_sample : k_plain;
+  int32_t* __restrict__ topk_idx = sample ? out_sample : out_plain;
   const int tid = threadIdx.x, lane = tid & 31;
   const float* rowp = logits + static_cast<size_t>(row) * V;
   const float* rowg = kSample ? gumbel + static_cast<size_t>(row) * V : nullptr;
@@ -112,7 +119,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
         float4 t = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
         if (i0 < part_end) {
           t = __ldcs(reinterpret_cast<const float4*>(rowp + i0));
-          if (kSample) {
+          if (kSample && sample) {
             const float4 g = __ldcs(reinterpret_cast<const float4*>(rowg + i0));
             t.x = __fadd_rn(__fmul_rn(t.x, inv_t), g.x); t.y = __fadd_rn(__fmul_rn(t.y, inv_t), g.y);
             t.z = __fadd_rn(__fmul_rn(t.z, inv_t), g.z); t.w = __fadd_rn(__fmul_rn(t.w, inv_t), g.w);
@@ -127,7 +134,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
         float x = -INFINITY;
         if (i < part_end) {
           x = __ldcs(rowp + i);
-          if (kSample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcs(rowg + i));
+          if (kSample && sample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcs(rowg + i));
         }
         v[j] = x;
       }
@@ -240,7 +247,7 @@ tr_topk_kernel(const float* __restrict__ logits, int V, int k, int chunks_per_pa
       u64 best = 0;
       for (int i = part_base + tid; i < part_end; i += KT) {
         float x = __ldcg(rowp + i);
-        if (kSample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcg(rowg + i));
+        if (kSample && sample) x = __fadd_rn(__fmul_rn(x, inv_t), __ldcg(rowg + i));
         const u64 key = topk_key(x, i);
         if (key < last && key > best) best = key;
       }
@@ -315,18 +322,21 @@ extern "C" int tr_debug_stamps_topk(unsigned long long* host, int reset) {
 #endif
 
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
-                         const float* d_gumbel, float inv_temperature, int k_override) {
+                         const float* d_gumbel, float inv_temperature, int32_t* d_drawn) {
+  // without noise: the rows' top-k.  With noise: the same launch also holds one more cluster per row that ranks
+  // logit * inv_temperature + noise and writes its first entry (the draw) to d_drawn.
   const int rows = ctx->batch * ctx->n_nodes;
-  const int k = k_override > 0 ? k_override : ctx->k;
+  const int k = ctx->k;
   const int chunks = (ctx->vocab + CHUNK - 1) / CHUNK;
   int P = 1;
   while (P < MAX_PARTS && P < chunks) P *= 2;
   const int cpp = (chunks + P - 1) / P;
   bool vec = (ctx->vocab % 4 == 0) && ((reinterpret_cast<uintptr_t>(d_logits) & 15) == 0);
   if (d_gumbel) vec = vec && ((reinterpret_cast<uintptr_t>(d_gumbel) & 15) == 0);
+  if (d_gumbel && (!d_drawn || 2 * rows > 65535)) return TR_ERR_UNSUPPORTED;
 
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(P, rows);
+  cfg.gridDim = dim3(P, d_gumbel ? 2 * rows : rows);
   cfg.blockDim = dim3(KT);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = s;
@@ -342,11 +352,15 @@ tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx
   const int V = ctx->vocab;
   cudaError_t e;
   if (d_gumbel)
-    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, inv_temperature)
-            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, inv_temperature);
+    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel,
+                                 inv_temperature, rows, 1, d_drawn)
+            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, true>, d_logits, V, k, cpp, d_topk_idx, d_gumbel,
+                                 inv_temperature, rows, 1, d_drawn);
   else
-    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f)
-            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f);
+    e = vec ? cudaLaunchKernelEx(&cfg, tr_topk_kernel<true, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f, rows, 1,
+                                 d_drawn)
+            : cudaLaunchKernelEx(&cfg, tr_topk_kernel<false, false>, d_logits, V, k, cpp, d_topk_idx, d_gumbel, 1.f, rows, 1,
+                                 d_drawn);
   TR_CUDA_TRY(e);
   return TR_OK;
 }

@@ -286,12 +286,9 @@ extern "C" tr_status tr_verify_update_sampled(tr_ctx* ctx, const float* d_logits
     return TR_ERR_INVALID_ARG;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   int32_t* drawn = d_sampled ? d_sampled : ctx->d_sampled;
-  // the candidates stored in the matrix are the model's top-k, whatever is drawn
-  tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s);
-  if (st != TR_OK) return st;
-  // the draw: the first entry of the same ranking applied to logit / T + noise (the scratch lists are reused: the
-  // kernels are ordered on the stream)
-  st = tr_launch_topk(ctx, d_logits, drawn, s, d_gumbel, inv_temperature, 1);
+  // one launch, two clusters per row: the model's top-k (the candidates stored in the matrix, whatever is drawn) and
+  // the draw - the first entry of the same ranking applied to logit / T + noise
+  tr_status st = tr_launch_topk(ctx, d_logits, out->d_topk_idx, s, d_gumbel, inv_temperature, drawn);
   if (st != TR_OK) return st;
   return tr_launch_tail(ctx, d_tree, out, s, drawn, true);
 }

@@ -110,10 +110,10 @@ __device__ __forceinline__ unsigned long long tr_globaltimer() {
 #endif
 
 // launchers (host functions defined next to their kernels)
-// With d_gumbel: the kernel ranks z = fl32(fl32(logit * inv_temperature) + gumbel) instead of the logits, k_override
-// entries per row (1: the draw of temperature sampling).
+// With d_gumbel: the same launch also draws one token per row - the first entry of the ranking of
+// z = fl32(fl32(logit * inv_temperature) + gumbel) - into d_drawn [batch * N] (temperature sampling).
 tr_status tr_launch_topk(tr_ctx* ctx, const float* d_logits, int32_t* d_topk_idx, cudaStream_t s,
-                         const float* d_gumbel = nullptr, float inv_temperature = 1.f, int k_override = 0);
+                         const float* d_gumbel = nullptr, float inv_temperature = 1.f, int32_t* d_drawn = nullptr);
 // d_target [batch, N] (optional): the token every node's children are matched against, instead of topk[:, 0]
 // tree_early: d_tree was written at least two kernels back on the stream (the kernel directly in front did not write it)
 tr_status tr_launch_tail(tr_ctx* ctx, const int32_t* d_tree, const tr_step_out* out, cudaStream_t s,
