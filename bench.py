@@ -180,7 +180,7 @@ def run_reference(args, w):
 # ---------------------------------------------------------------------------------------------------
 def measure_lm_head(torch, tr, dw, w, dev, reps=20):
     """The output layer fused with argtopk (not part of the timed step, whose logits come from the toy model): one
-    pass over a random bf16 weight [V, hidden] for the step's batch * N rows, as a CUDA graph replayed `reps` times.
+    pass over a random bf16 weight [V, hidden] for the step's batch * N rows; graphs of 4 calls, `reps` calls in all.
     The weight (hundreds of MB) is larger than L2, so every replay streams it from HBM."""
     H = w.n_q_heads * w.head_dim
     rows = w.batch * w.n_nodes
@@ -192,19 +192,22 @@ def measure_lm_head(torch, tr, dw, w, dev, reps=20):
     graph = torch.cuda.CUDAGraph()
     tr.tr_lm_head_topk(dw.ctx, d_h, d_w, idx)
     torch.cuda.synchronize()
+    per_graph = 4                                              # calls per graph, like the steps of a round graph
     with torch.cuda.stream(s):
         with torch.cuda.graph(graph, stream=s):
-            tr.tr_lm_head_topk(dw.ctx, d_h, d_w, idx, stream=s)
+            for _ in range(per_graph):
+                tr.tr_lm_head_topk(dw.ctx, d_h, d_w, idx, stream=s)
     for _ in range(3):
         graph.replay()
     torch.cuda.synchronize()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n_rep = max(1, reps // per_graph)
     e0.record()
-    for _ in range(reps):
+    for _ in range(n_rep):
         graph.replay()
     e1.record()
     torch.cuda.synchronize()
-    us = e0.elapsed_time(e1) / reps * 1000.0
+    us = e0.elapsed_time(e1) / (n_rep * per_graph) * 1000.0
     groups = (rows + 127) // 128                               # row groups: the CTAs of a vocabulary slice share it via L2
     byts = w.vocab * H * 2 + rows * H * 2 + rows * w.k * 4      # algorithmic: the weight ONCE, hidden states, output
     return {"us": us, "bound": "hbm", "achieved": byts / us / 1e3, "unit": "GB/s", "algorithmic_bytes": byts,
