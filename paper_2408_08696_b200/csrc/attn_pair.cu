@@ -479,16 +479,18 @@ tr_attn_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
               __nv_bfloat162 pk = __floats2bfloat162_rn(p0, p1);
               preg[(q & 1) * 16 + (cc >> 1)] = *reinterpret_cast<uint32_t*>(&pk);
             }
+          // The other stream's turn begins when this stream's last exponentials are done: its softmax starts with work
+          // that does not need the special-function unit (TMEM loads, the maximum), which so runs under this stream's
+          // last P store (2 % faster than handing over after the store; handing over earlier still - with up to a quarter
+          // of the exponentials to go - measured the same, after the first half slower).
+          if (h == 1 && x.ns == 2 && lane == 0) mbar_arrive(bar(BAR_TURN + (s ^ 1)));
           tc_st32(s_col(s) + lane_base + h * 32u, preg);
           tc_wait_st();
           tc_fence_before();
           __syncwarp();
           if (lane == 0) mbar_arrive(bar(BAR_PFULL + 2 * s + h));
         }
-        if (x.ns == 2) {  // the other stream's turn (handing over after the first half already measured slower)
-          if (lane == 0) mbar_arrive(bar(BAR_TURN + (s ^ 1)));
-          ++gp;
-        }
+        if (x.ns == 2) ++gp;
         float se, so;
         unpack2(add2(add2(sm2[0], sm2[1]), add2(sm2[2], sm2[3])), se, so);
         l += se + so;
