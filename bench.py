@@ -550,6 +550,10 @@ NCU_TRAFFIC_BYTES = {
     # profiles/tr_attn_pair_kernel_llama3-8b_12layers.md: (414.64 MB read + 3.81 MB written) per 12-layer launch,
     # scaled to 32 layers
     "llama3-8b": int(round(32 / 12 * (414_638_080 + 3_806_208))),
+    # profiles/tr_attn_tc_kernel_llama2-13b_4layers.md: (345.53 MB read + 3.08 MB written) per 4-layer launch, 40 layers
+    "llama2-13b": 10 * (345_531_392 + 3_084_032),
+    # profiles/tr_attn_pair_kernel_llama2-70b-b8_4layers.md: (365.11 MB read + 4.73 MB written) per 4-layer launch, 80 layers
+    "llama2-70b-b8": 20 * (365_111_040 + 4_734_720),
 }
 
 
