@@ -160,12 +160,22 @@ def test_loop_llama2_7b_shape(harness):
     _run_loop(harness, synth.WORKLOADS["llama2-7b"], 24)
 
 
+def test_loop_llama2_7b_all_256_steps_of_the_workload_as_graph_replays(harness):
+    """The benchmark's workload from its first step to its last (256 steps, the replayed single-step graphs): every
+    integer output of every step and the matrix at the end, bit for bit.  About a minute of oracle time."""
+    _run_loop(harness, synth.WORKLOADS["llama2-7b"], 256, graphs=True)
+
+
 def test_loop_batched_8_sequences_via_graph(harness):
     _run_loop(harness, synth.WORKLOADS["llama2-70b-b8"], 12, graphs=True)
 
 
 def test_loop_large_vocab(harness):
     _run_loop(harness, synth.WORKLOADS["llama3-8b"], 6)
+
+
+def test_loop_large_vocab_32_steps_as_graph_replays(harness):
+    _run_loop(harness, synth.WORKLOADS["llama3-8b"], 32, graphs=True)
 
 
 @pytest.mark.parametrize("rule,only_accepted", [("first", False), ("last", True), ("first", True)])
