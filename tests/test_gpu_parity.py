@@ -441,6 +441,19 @@ def test_loop_template_breadth_and_depth_sweep(harness, branching, n_nodes, k, b
     assert 1.0 <= mat <= max(orc.node_depth(parent)) + 1          # Appendix: at most depth + 1 tokens per step
 
 
+@pytest.mark.parametrize("hq,hkv,head_dim,ctx,splits", [
+    (2, 2, 128, 30000, 0),      # 235 key tiles per unit, split along the keys over the SMs + merge
+    (2, 2, 128, 30000, 1),      # ... and as one unit per head: 235 tiles through one CTA's ring
+    (8, 2, 128, 30000, 1),      # the two-tiles-per-CTA kernel on a long stream
+    (2, 1, 64, 33000, 0),       # head_dim 64, a prefix longer than 2^15 keys
+])
+def test_attention_long_context(harness, hq, hkv, head_dim, ctx, splits):
+    """Prefixes of 30 000 and more keys (hundreds of key tiles per unit: ring wrap-arounds, barrier phases, the running
+    maximum over a long row), one layer, every head against the oracle."""
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=hq, n_kv_heads=hkv, head_dim=head_dim, ctx=(ctx,))
+    _attention_case(harness, w, 1, splits=splits)
+
+
 def test_attention_single_node_tree(harness):
     w = dataclasses.replace(synth.WORKLOADS["tiny"], n_nodes=1, branching=(1,), ctx=(50,))
     _attention_case(harness, w, 1)
