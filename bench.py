@@ -428,7 +428,8 @@ def run_ours(args, w):
     per_layer_ms = None
     if dw.L > 1:
         args_l = [tr.make_attn_args(dw.ctx, dw.q[:, l:l + 1], dw.k[:, l:l + 1], dw.v[:, l:l + 1], dw.o[:, l:l + 1],
-                                    dw.d_ctx_len, w.max_ctx) for l in range(dw.L)]
+                                    dw.d_ctx_len, w.max_ctx, prefix_stable=True) for l in range(dw.L)]
+        # (prefix_stable: nothing writes the prefix lengths or the prefix K/V between these launches)
         gl = torch.cuda.CUDAGraph()
         s2 = torch.cuda.Stream(dev)
         with torch.cuda.stream(s2):

@@ -117,6 +117,14 @@ tr_status tr_build_tree(tr_ctx* ctx, const int32_t* d_root, int32_t* d_tree, voi
  * this is for callers that hold all layers' q already, e.g. benchmarks).
  * The call uses scratch of the context (split-KV partials, a unit counter): calls on one context must not overlap
  * on the device (one stream, or streams ordered by events).
+ * Early start (prefix_stable != 0).  A short launch (fewer units than SMs, e.g. one layer of one sequence) is split
+ * along the keys and launched so that it may begin while the kernel in front of it on the stream is still draining.
+ * By default it touches no global memory until that kernel has finished.  With prefix_stable the caller vouches that
+ * d_ctx_len and the cache rows below C_b (the prefix) are NOT written by the kernel directly in front of this call
+ * (nor by a kernel that this one let start early before its own inputs were complete): the launch then requests its
+ * prefix K/V tiles at once and only q, the tree's K/V rows and the output wait.  True for the usual caller - the
+ * kernel in front writes this layer's q and tree rows - and false directly behind tr_commit, which moves rows into
+ * the prefix and changes d_ctx_len.  Ignored by launches that are not split.
  * Errors: TR_ERR_INVALID_ARG (NULL, bad head counts, alignment), TR_ERR_UNSUPPORTED (head_dim not 64/128).
  */
 typedef struct {
@@ -133,6 +141,7 @@ typedef struct {
   int64_t layer_stride_q, layer_stride_kv, layer_stride_o;
   float scale;    /* 0 -> 1/sqrt(head_dim) */
   int32_t splits; /* 0 -> chosen by the library; >0 forces that many KV splits (testing) */
+  int32_t prefix_stable; /* non-zero: see above ("Early start") */
 } tr_attn_args;
 tr_status tr_tree_attention(tr_ctx* ctx, const tr_attn_args* args, void* stream);
 

@@ -46,7 +46,7 @@ class tr_attn_args(C.Structure):
         ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
         ("n_layers", C.c_int32),
         ("layer_stride_q", C.c_int64), ("layer_stride_kv", C.c_int64), ("layer_stride_o", C.c_int64),
-        ("scale", C.c_float), ("splits", C.c_int32),
+        ("scale", C.c_float), ("splits", C.c_int32), ("prefix_stable", C.c_int32),
     ]
 
 
@@ -201,7 +201,7 @@ def tr_build_tree(ctx, d_root, d_tree, stream=None):
                              _stream(stream)), "tr_build_tree")
 
 
-def make_attn_args(ctx, q, k_cache, v_cache, out, d_ctx_len, max_ctx, scale=0.0, splits=0):
+def make_attn_args(ctx, q, k_cache, v_cache, out, d_ctx_len, max_ctx, scale=0.0, splits=0, prefix_stable=False):
     """q/out: bf16 [B, L, N, Hq, D]; k_cache/v_cache: bf16 [B, L, Hkv, R, D]; d_ctx_len int32 [B].
     Any strides with a contiguous last dimension are passed through."""
     a = tr_attn_args()
@@ -224,6 +224,7 @@ def make_attn_args(ctx, q, k_cache, v_cache, out, d_ctx_len, max_ctx, scale=0.0,
     a.n_layers = L
     a.layer_stride_q, a.layer_stride_kv, a.layer_stride_o = q.stride(1), k_cache.stride(1), out.stride(1)
     a.scale, a.splits = float(scale), int(splits)
+    a.prefix_stable = 1 if prefix_stable else 0
     return a
 
 

@@ -48,6 +48,7 @@ struct TcParams {
   // are packed into common 128-row tiles (row = node * G + head-in-group), MT tiles per head unit; when the group
   // size does not divide 128, every query head is its own head unit (G = 1) and kv_div maps it to its KV head.
   int HU, G, g_shift, MT, kv_div;
+  int early_prefix;  // the producer may fetch prefix K/V tiles before it waits for the kernel in front (see tr.h)
   int live_warps;  // softmax warps that own at least one real row in every unit (4 unless tiles are unpacked and N <= 96)
   uint32_t div_MT[2], div_S[2], div_HU[2], div_L[2], div_kv[2];  // (multiplier, shift) for exact u32 division
   int64_t os_b, os_h, os_t, os_l;
@@ -192,7 +193,9 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
   };
   if (!kPdl) stage_ctx_len();
 
-  if (tid == 0) {
+  // (the TMA producer's thread sets the barriers up, so that it can start copying before the CTA's first barrier)
+  uint32_t c_early = 0;  // producer only: ring entries of the first unit issued before the dependency wait
+  if (tid == WARP_PRODUCER * 32) {
     for (int i = 0; i < NST_MAX; ++i) { mbar_init(bar(BAR_FULL + i), 1); mbar_init(bar(BAR_EMPTY + i), 1); }
     for (int i = 0; i < 2; ++i) {
       mbar_init(bar(BAR_QFULL + i), 1);
@@ -207,6 +210,34 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     *s_abort = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (kPdl && p.early_prefix) {
+      // The caller vouches that the prefix lengths and the prefix rows of the caches are not being written by
+      // whatever still runs in front of this launch: the K/V tiles of this CTA's first unit that lie wholly inside
+      // the prefix are requested now, under the tail of the kernel in front; Q and the tiles that reach into the
+      // tree's rows follow after the wait.
+      const int nb = p.n_units / (p.L * p.HU * p.S * p.MT);
+      for (int i = 0; i < nb && i < CTX_CACHE; ++i) s_ctx[i] = __ldcg(p.ctx_len + i);
+      const uint64_t pol = l2_policy_evict_first();
+      int u = blockIdx.x;
+      Unit x = decode_unit(p, u, s_ctx);
+      while (x.t0 >= x.t1 && u + static_cast<int>(gridDim.x) < p.n_units) { u += gridDim.x; x = decode_unit(p, u, s_ctx); }
+      if (x.t0 < x.t1) {
+        const int t_end = min(x.t1, x.C / BK);  // tiles below hold prefix keys only
+        for (int t = x.t0; t < t_end && c_early + 2u <= static_cast<uint32_t>(NST); ++t) {
+#pragma unroll
+          for (int kv = 0; kv < 2; ++kv) {
+            const uint32_t slot = c_early % NST;
+            const CUtensorMap* m = kv == 0 ? &map_k : &map_v;
+            const uint32_t dst = base + SM_RING + slot * TILE_BYTES;
+            mbar_expect_tx(bar(BAR_FULL + slot), TILE);
+            tma_load_5d_hint(dst, m, bar(BAR_FULL + slot), 0, t * BK, x.kvh, x.layer, x.b, pol);
+            if (NBOX == 2)
+              tma_load_5d_hint(dst + BOX_BYTES, m, bar(BAR_FULL + slot), 64, t * BK, x.kvh, x.layer, x.b, pol);
+            ++c_early;
+          }
+        }
+      }
+    }
   }
   if (warp == WARP_MMA) {  // TMEM: all 512 columns (one CTA per SM)
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(base + SM_MISC), "r"(512u)
@@ -249,6 +280,7 @@ tr_attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int t = x.t0; t < x.t1 && ok; ++t) {
 #pragma unroll
           for (int kv = 0; kv < 2; ++kv) {
+            if (c < c_early) { ++c; continue; }  // requested before the dependency wait
             const uint32_t slot = c % NST, par = ((c / NST) & 1u) ^ 1u;
             ok = mbar_wait(bar(BAR_EMPTY + slot), par, s_abort);
             if (!ok) break;
@@ -598,6 +630,9 @@ bool encode_map(CUtensorMap* m, const void* ptr, const uint64_t (&dims)[5], cons
 // units: (((b, layer, head unit), split), tile).
 __global__ void __launch_bounds__(256) tr_attn_tc_combine_kernel(const TcParams p) {
   tr_grid_dependency_wait();  // launched with programmatic dependent launch: the partials come from the kernel before
+  // the kernel behind this one may be scheduled now (it waits for this grid before it reads what is written here);
+  // a following attention launch uses the time to set itself up and, if allowed, to request prefix K/V
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int r = blockIdx.x * 8 + (threadIdx.x >> 5);  // row of the tile
   const int d = (threadIdx.x & 31) * 4;
   if (d >= p.HD) return;                              // head_dim 64: half the lanes have no column
@@ -697,6 +732,7 @@ tr_status tr_launch_attention_tc(tr_ctx* ctx, const tr_attn_args* a, cudaStream_
   p.HU = packed ? a->n_kv_heads : a->n_q_heads;
   p.kv_div = packed ? 1 : group;
   p.MT = (ctx->n_nodes * p.G + 127) / 128;
+  p.early_prefix = a->prefix_stable ? 1 : 0;
   p.live_warps = (p.MT == 1 && p.G == 1) ? (ctx->n_nodes + 31) / 32 : 4;
   const int64_t base = static_cast<int64_t>(ctx->batch) * a->n_layers * p.HU * p.MT;
   if (base > (1 << 30)) return TR_ERR_UNSUPPORTED;

@@ -454,6 +454,48 @@ def test_attention_long_context(harness, hq, hkv, head_dim, ctx, splits):
     _attention_case(harness, w, 1, splits=splits)
 
 
+@pytest.mark.parametrize("hq,hkv,ctxs", [(32, 32, (1024,)), (8, 2, (300, 77)), (4, 4, (50,))])
+def test_attention_per_layer_launches_with_early_prefix_requests(harness, tr, hq, hkv, ctxs):
+    """One launch per layer, back to back on a stream and as a replayed graph, with the caller's promise that prefix
+    lengths and prefix K/V are stable (prefix_stable): a launch may then request its prefix tiles while the launch in
+    front (the previous layer's merge of split partials) is still running.  Every head of every layer against the
+    oracle; the outputs must not depend on the promise."""
+    L = 4
+    w = dataclasses.replace(synth.WORKLOADS["llama2-7b"], n_q_heads=hq, n_kv_heads=hkv, ctx=ctxs)
+    dw = harness.DeviceWorkload(w, n_layers=L)
+    q, k, v = synth.attention_inputs(w, L)
+    ref = [[oracle_attention(w, q, k, v, b, l, dw.parent) for l in range(L)] for b in range(w.batch)]
+
+    def check():
+        torch.cuda.synchronize()
+        got = dw.o.float().cpu().numpy()
+        for b in range(w.batch):
+            for l in range(L):
+                for h in range(hq):
+                    mx, rel = attention_close(got[b, l, :, h], ref[b][l][:, h])
+                    assert mx <= ATOL and rel <= RTOL, (b, l, h, mx, rel)
+
+    for stable in (False, True):
+        args = [tr.make_attn_args(dw.ctx, dw.q[:, l:l + 1], dw.k[:, l:l + 1], dw.v[:, l:l + 1], dw.o[:, l:l + 1],
+                                  dw.d_ctx_len, w.max_ctx, prefix_stable=stable) for l in range(L)]
+        dw.o.zero_()
+        for a in args:
+            tr.tr_tree_attention(dw.ctx, a)
+        check()
+        s = torch.cuda.Stream(dw.dev)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(s):
+            with torch.cuda.graph(g, stream=s):
+                for a in args:
+                    tr.tr_tree_attention(dw.ctx, a, s)
+        for _ in range(3):
+            dw.o.zero_()
+            g.replay()
+            check()
+    assert tr.tr_device_flags(dw.ctx) == 0
+    dw.close()
+
+
 def test_attention_single_node_tree(harness):
     w = dataclasses.replace(synth.WORKLOADS["tiny"], n_nodes=1, branching=(1,), ctx=(50,))
     _attention_case(harness, w, 1)
