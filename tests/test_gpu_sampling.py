@@ -95,3 +95,23 @@ def test_sampling_argument_errors(harness, tr):
         with pytest.raises(tr.TrError):
             tr.tr_verify_update_sampled(dw.ctx, dw.d_logits[0], d_g, bad, dw.d_tree, dw.out_struct)
     dw.close()
+
+
+def test_sampling_rejects_more_rows_than_one_launch_can_hold(tr):
+    """The top-k and the draw of a row are two clusters of one launch: 2 * batch * N must fit into the grid's second
+    dimension.  A batch that tr_init accepts (batch * N <= 65535) but that is too large for the sampled call gets
+    TR_ERR_UNSUPPORTED before anything is launched; the greedy call still works."""
+    n, batch, V, k = 80, 410, 16, 1                      # 32 800 rows: 2 x that is more than 65 535
+    parent, rank = tr.tr_template_from_branching((1,), n)
+    ctx = tr.tr_init(V, k, parent, rank, batch=batch)
+    out_struct, out = tr.make_step_out(ctx)
+    d_logits = torch.zeros(batch, n, V, device="cuda")
+    d_logits[:, :, 3] = 1.0
+    d_tree = torch.zeros(batch, n, dtype=torch.int32, device="cuda")
+    with pytest.raises(tr.TrError) as e:
+        tr.tr_verify_update_sampled(ctx, d_logits, torch.zeros_like(d_logits), 1.0, d_tree, out_struct)
+    assert e.value.status == tr.TR_ERR_UNSUPPORTED
+    tr.tr_verify_update(ctx, d_logits, d_tree, out_struct)
+    torch.cuda.synchronize()
+    assert (out["topk_idx"].cpu().numpy() == 3).all() and tr.tr_device_flags(ctx) == 0
+    tr.tr_destroy(ctx)
