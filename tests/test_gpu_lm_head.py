@@ -64,6 +64,7 @@ CASES = {
     "two-row-groups": (_wl(ctx=(128, 128, 128, 128, 128, 128, 128, 128, 128, 128, 128)), None),  # 165 rows > 128
     "llama3-vocab-chunks": (_wl("llama3-8b", n_q_heads=2, n_kv_heads=2), None),   # 128256 tokens: 4 chunks per CTA
     "llama2-7b": (_wl("llama2-7b"), None),                           # the bench shape: 80 x 4096 x 32000
+    "llama2-70b-b8": (_wl("llama2-70b-b8"), None),                   # 640 rows = 5 row groups side by side, hidden 8192
 }
 
 
