@@ -305,9 +305,23 @@ def check_parity(torch, tr, harness, dw, w, graphs, round_graph):
     return res
 
 
+def ensure_built():
+    """The product path needs the CUDA library (there is no fallback).  Local rank 0 builds it if it is missing or
+    older than its sources; the other ranks of the node wait for the files."""
+    from paper_2408_08696_b200 import build
+    if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+        build.build()
+        return
+    deadline = time.time() + 600
+    while time.time() < deadline and not (os.path.exists(build.LIB_TR) and os.path.exists(build.LIB_SYNTH)):
+        time.sleep(1.0)
+    time.sleep(2.0)  # (a library that is being rewritten: let rank 0's linker finish)
+
+
 def run_ours(args, w):
     import torch
     import torch.distributed as dist
+    ensure_built()
     from paper_2408_08696_b200 import binding as tr
     from paper_2408_08696_b200 import harness, replicas, synth
 
@@ -577,6 +591,7 @@ def main():
     w = synth.WORKLOADS[args.workload]
     if args.lm_head_only:
         import torch
+        ensure_built()
         from paper_2408_08696_b200 import binding as tr
         from paper_2408_08696_b200 import harness
         dw = harness.DeviceWorkload(w, with_attention=False)
